@@ -1,0 +1,420 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU, no CUDA library).
+
+Each test checks the oracle against something other than itself: a closed form, an invariant, a
+textbook special case, brute force on a tiny input, or a value the paper prints.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import esparse_oracle as orc
+from paper_2310_15929_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def golden():
+    out = {}
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, *v = line.split()
+                out[k] = [float(x) for x in v]
+    return out
+
+
+def rand_layer(seed, No, C, T, outliers=2):
+    g = np.random.default_rng(seed)
+    W = (g.standard_normal((No, C)) * 0.02).astype(np.float16)
+    X = g.standard_normal((T, C))
+    X[:, g.choice(C, outliers, replace=False)] *= 20
+    return W, X.astype(np.float16)
+
+
+# Independent naive restatements used only here -------------------------------------------------
+def naive_objective(W, s, theta):
+    """Eq. 5 written directly on the full metric matrix: sort every group, add its 2 largest."""
+    xi = np.abs(W.astype(np.float64)) * s[None, :]
+    xp = xi[:, theta].reshape(W.shape[0], -1, 4)
+    return float(np.sort(xp, axis=2)[:, :, 2:].sum())
+
+
+def naive_mask_top2(score_matrix):
+    """Textbook 2:4 magnitude-style mask on a [No, C] score matrix, identity order; ties -> lower index."""
+    No, C = score_matrix.shape
+    m = np.zeros((No, C), dtype=bool)
+    for j in range(No):
+        for g in range(C // 4):
+            v = score_matrix[j, 4 * g:4 * g + 4]
+            order = sorted(range(4), key=lambda k: (-v[k], k))
+            for k in order[:2]:
+                m[j, 4 * g + k] = True
+    return m
+
+
+# ------------------------------------------------------------------------------------------ paper constants
+def test_paper_constants_consistent():
+    g = golden()
+    assert orc.BINS == int(g["entropy_bins"][0])
+    assert orc.LBS_BLOCK == int(g["lbs_block"][0])
+    # C! orderings of 1024 channels ~ 10^2640
+    log10_fact = math.lgamma(int(g["orderings_channels"][0]) + 1) / math.log(10)
+    assert abs(log10_fact - g["orderings_log10"][0]) < 1.0
+    # Table 6 rows are self-consistent and approach the per-layer closed form 1 - 9/16 from below
+    for d, s_, pct in zip(g["mem_dense_gb"], g["mem_sparse_gb"], g["mem_saving_pct"]):
+        assert abs((1 - s_ / d) * 100 - pct) < 0.06
+        assert pct < 43.75
+    assert g["mem_saving_pct"] == sorted(g["mem_saving_pct"])
+    # speedup = 1 / (1 - latency reduction)
+    for red, sp in zip(g["latency_reduction_pct"], g["speedup"]):
+        assert abs(1 / (1 - red / 100) - sp) < 0.01
+
+
+# ------------------------------------------------------------------------------------------ O1 norm
+def test_norm_closed_form_constant_channel():
+    T = 4096
+    X = np.full((T, 3), 0.5, dtype=np.float16)
+    X[:, 1] = -3.0
+    X[:, 2] = 0.0
+    assert np.array_equal(orc.channel_norm(X), np.array([0.5 * 64, 3.0 * 64, 0.0]))
+
+
+def test_norm_matches_library_and_invariances():
+    _, X = rand_layer(1, 8, 64, 777)
+    am = orc.channel_norm(X)
+    ref = np.linalg.norm(X.astype(np.float64), axis=0)
+    assert np.allclose(am, ref, rtol=1e-13, atol=0)
+    # exact power-of-two scaling, token permutation
+    assert np.array_equal(orc.channel_norm(X * np.float16(4.0)), am * 4.0)
+    perm = np.random.default_rng(2).permutation(X.shape[0])
+    assert np.allclose(orc.channel_norm(X[perm]), am, rtol=1e-14, atol=0)
+    # 3-4-5 triangle
+    assert orc.channel_norm(np.array([[3.0], [4.0]], dtype=np.float16))[0] == 5.0
+
+
+# ------------------------------------------------------------------------------------------ O2 entropy
+def test_entropy_uniform_spread_is_log_bins():
+    # T = 100 r values equally spread over the range: every one of the 100 bins gets r of them.
+    r = 3
+    vals = np.repeat(np.arange(100, dtype=np.float64), r)     # 0..99, exact in fp16
+    vals = np.concatenate([vals[:-1], [99.0]])
+    X = np.random.default_rng(0).permutation(vals)[:, None].astype(np.float16)
+    # range [0, 99]: bin = floor(x * 100 / 99) = x for x < 99, and the maximum is clamped into bin 99
+    counts = orc.channel_histogram(X)
+    assert np.array_equal(counts[0], np.full(100, r))
+    assert abs(orc.channel_entropy(X)[0] - math.log(100)) < 1e-14
+
+
+def test_entropy_constant_two_valued_and_bounds():
+    T = 64
+    X = np.zeros((T, 4), dtype=np.float16)
+    X[:, 0] = 7.0                       # constant -> 0
+    X[: T // 2, 1] = -1.0               # half / half -> ln 2
+    X[T // 2:, 1] = 2.0
+    X[: T // 4, 2] = 1.0                # quarter / three quarters
+    g = np.random.default_rng(3)
+    X[:, 3] = g.standard_normal(T).astype(np.float16)
+    ir = orc.channel_entropy(X)
+    assert ir[0] == 0.0
+    assert abs(ir[1] - math.log(2)) < 1e-15
+    assert abs(ir[2] - (-(0.25 * math.log(0.25) + 0.75 * math.log(0.75)))) < 1e-15
+    assert 0.0 <= ir[3] <= math.log(min(100, T)) + 1e-12
+    counts = orc.channel_histogram(X)
+    assert np.all(counts.sum(axis=1) == T)
+    assert counts[3, 0] >= 1 and counts[3, 99] >= 1        # min in first bin, max in last
+
+
+def test_entropy_affine_invariance_and_token_order():
+    g = np.random.default_rng(4)
+    X = (g.integers(-200, 200, size=(500, 6)) / 8.0).astype(np.float16)   # exactly representable
+    ir = orc.channel_entropy(X)
+    assert np.array_equal(orc.channel_entropy(X * np.float16(4.0)), ir)
+    assert np.array_equal(orc.channel_entropy((X + np.float16(16.0)).astype(np.float16)), ir)
+    assert np.array_equal(orc.channel_histogram(X[g.permutation(500)]), orc.channel_histogram(X))
+    # negation mirrors the bins except at bin edges; entropy equal when no value sits on an interior edge
+    c = orc.channel_histogram(X)
+    assert c.sum() == 500 * 6
+
+
+def test_bin_index_against_exact_rational_arithmetic():
+    from fractions import Fraction
+    g = np.random.default_rng(5)
+    X = g.standard_normal((300, 5)).astype(np.float16)
+    counts = orc.channel_histogram(X)
+    for c in range(5):
+        col = [Fraction(float(v)) for v in X[:, c]]
+        lo, hi = min(col), max(col)
+        ref = np.zeros(100, dtype=np.int64)
+        for v in col:
+            ref[min(99, int(((v - lo) * 100) // (hi - lo)))] += 1   # floor of the exact quotient
+        assert np.array_equal(counts[c], ref)
+
+
+# ------------------------------------------------------------------------------------------ O3 score / metric
+def test_score_toggles_and_norm_only_baseline():
+    W, X = rand_layer(6, 16, 32, 200)
+    am, ir = orc.channel_norm(X), orc.channel_entropy(X)
+    assert np.array_equal(orc.channel_score(ir, am, 0.5), ir + 0.5 * am)
+    assert np.array_equal(orc.channel_score(ir, am, 0.5, use_entropy=False), 0.5 * am)
+    assert np.array_equal(orc.channel_score(ir, am, 0.5, use_norm=False), ir)
+    # entropy off => the metric is |w| * alpha * ||x||_2: masks equal a textbook top-2 of |W| * norm
+    s = orc.channel_score(ir, am, 1.0, use_entropy=False)
+    vals, meta, _ = orc.select_compress(W, s, np.arange(32))
+    mask = orc.decompress_permuted(np.ones_like(vals), meta) != 0
+    ref = naive_mask_top2(np.abs(W.astype(np.float64)) * np.linalg.norm(X.astype(np.float64), axis=0)[None, :])
+    assert np.array_equal(mask, ref)
+    assert np.array_equal(orc.metric(W, s), np.abs(W.astype(np.float64)) * s[None, :])
+
+
+def test_zero_score_falls_back_to_position_tiebreak():
+    W = np.random.default_rng(7).standard_normal((4, 16)).astype(np.float16)
+    X = np.ones((10, 16), dtype=np.float16)                 # constant channels: entropy 0
+    r = orc.metric_prune(W, X, alpha=0.0, use_lbs=False)
+    assert np.all(r.score == 0)
+    assert np.all(r.meta == 0x44)                            # positions 0,1 kept in every group
+    assert np.array_equal(r.theta0, orc.global_naive_shuffle(np.zeros(16))[0])
+
+
+# ------------------------------------------------------------------------------------------ O4 global shuffle
+def test_gns_closed_form_descending_means():
+    C = 8
+    theta0, near = orc.global_naive_shuffle(np.arange(C, 0, -1).astype(np.float64))
+    assert theta0.tolist() == [0, 2, 4, 6, 1, 3, 5, 7]      # groups {0,2,4,6}, {1,3,5,7}
+    assert near == 0
+    C = 64
+    G = C // 4
+    t, _ = orc.global_naive_shuffle(-np.arange(C, dtype=np.float64))
+    p = np.arange(C)
+    assert np.array_equal(t, (p % 4) * G + p // 4)
+
+
+def test_gns_bijection_quartiles_and_stability():
+    g = np.random.default_rng(8)
+    mean = g.random(256)
+    mean[10] = mean[200]                                      # a tie: lower index first
+    theta0, _ = orc.global_naive_shuffle(mean)
+    assert sorted(theta0.tolist()) == list(range(256))
+    rank = np.empty(256, dtype=np.int64)
+    rank[np.argsort(-mean, kind="stable")] = np.arange(256)
+    assert rank[10] + 1 == rank[200]
+    quart = rank[theta0].reshape(64, 4) // 64
+    assert np.all(np.sort(quart, axis=1) == np.arange(4)[None, :])   # one channel per rank quartile
+    assert np.all(np.abs(np.diff(np.sort(rank[theta0].reshape(64, 4), axis=1), axis=1)) == 64)
+
+
+def test_channel_mean_matches_plain_mean_of_metric():
+    W, X = rand_layer(9, 200, 48, 100)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.3)
+    assert np.allclose(orc.channel_mean_metric(W, s), orc.metric(W, s).mean(axis=0), rtol=1e-13, atol=0)
+    # exact column sums do not depend on the order of rows
+    assert np.array_equal(orc.channel_mean_metric(W[::-1], s), orc.channel_mean_metric(W, s))
+
+
+# ------------------------------------------------------------------------------------------ O5 block shuffle
+def test_objective_matches_naive_definition():
+    W, X = rand_layer(10, 64, 32, 80)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 1.0)
+    for seed in range(3):
+        theta = np.random.default_rng(seed).permutation(32).astype(np.int32)
+        assert abs(orc.objective(W, s, theta) - naive_objective(W, s, theta)) <= 1e-12 * naive_objective(W, s, theta)
+        assert abs(orc.group_value(W, s, theta[:4]) -
+                   np.sort(orc.metric(W, s)[:, theta[:4]], axis=1)[:, 2:].sum()) < 1e-10
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_lbs_invariants_and_local_optimality(seed):
+    W, X = rand_layer(20 + seed, 24, 32, 64)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.2)
+    theta0, _ = orc.global_naive_shuffle(orc.channel_mean_metric(W, s))
+    block = 16
+    theta, info = orc.local_block_shuffle(W, s, theta0, block=block)
+    assert sorted(theta.tolist()) == list(range(32))
+    for b in range(32 // block):                              # block-local with respect to theta0
+        assert sorted(theta[b * block:(b + 1) * block].tolist()) == sorted(theta0[b * block:(b + 1) * block].tolist())
+    assert naive_objective(W, s, theta) >= naive_objective(W, s, theta0)
+    # at exit no cross-group pair inside a block has positive gain (brute force on the naive objective)
+    base = naive_objective(W, s, theta)
+    for b in range(32 // block):
+        for i, j in itertools.combinations(range(b * block, (b + 1) * block), 2):
+            if i // 4 == j // 4:
+                continue
+            t2 = theta.copy()
+            t2[i], t2[j] = t2[j], t2[i]
+            assert naive_objective(W, s, t2) <= base * (1 + 1e-13)
+    # each applied swap strictly increases the objective: replay with a swap cap
+    prev = naive_objective(W, s, theta0)
+    for k in range(1, int(info.swaps_per_block.max()) + 1):
+        tk, _ = orc.local_block_shuffle(W, s, theta0, block=block, max_swaps=k)
+        cur = naive_objective(W, s, tk)
+        assert cur >= prev
+        prev = cur
+    assert abs(prev - base) <= 1e-12 * base
+
+
+def test_lbs_first_swap_is_the_best_pair_by_brute_force():
+    W, X = rand_layer(30, 40, 16, 50)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.1)
+    theta0 = np.arange(16, dtype=np.int32)
+    t1, info = orc.local_block_shuffle(W, s, theta0, block=16, max_swaps=1)
+    base = naive_objective(W, s, theta0)
+    best, arg = 0.0, None
+    for i, j in itertools.combinations(range(16), 2):
+        if i // 4 == j // 4:
+            continue
+        t2 = theta0.copy()
+        t2[i], t2[j] = t2[j], t2[i]
+        gain = naive_objective(W, s, t2) - base
+        if gain > best * (1 + 1e-9) + 1e-12:
+            best, arg = gain, (i, j)
+    if arg is None:
+        assert info.swaps_total == 0
+    else:
+        exp = theta0.copy()
+        exp[arg[0]], exp[arg[1]] = exp[arg[1]], exp[arg[0]]
+        assert np.array_equal(t1, exp)
+
+
+def test_lbs_vs_exhaustive_optimum_on_8_channels():
+    hits = 0
+    for seed in range(6):
+        W, X = rand_layer(40 + seed, 12, 8, 40, outliers=1)
+        s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.5)
+        theta0 = np.arange(8, dtype=np.int32)
+        theta, _ = orc.local_block_shuffle(W, s, theta0, block=8)
+        got = naive_objective(W, s, theta)
+        # only the split of the 8 channels into two groups of 4 matters: 35 distinct splits
+        best = max(naive_objective(W, s, np.array(list(a) + [c for c in range(8) if c not in a]))
+                   for a in itertools.combinations(range(8), 4))
+        assert got <= best * (1 + 1e-13)
+        one_swap = max(naive_objective(W, s, np.array(t)) for t in _one_swap_orders(theta0))
+        if abs(one_swap - best) <= 1e-13 * best:             # optimum one swap away => greedy reaches it
+            assert abs(got - best) <= 1e-12 * best
+            hits += 1
+        assert got >= one_swap * (1 - 1e-13) or got >= naive_objective(W, s, theta0)
+    assert hits >= 1
+
+
+def _one_swap_orders(theta0):
+    out = [theta0.copy()]
+    for i in range(4):
+        for j in range(4, 8):
+            t = theta0.copy()
+            t[i], t[j] = t[j], t[i]
+            out.append(t)
+    return out
+
+
+def test_lbs_incremental_equals_from_scratch_on_config0():
+    wl = inputs.WORKLOADS[0]
+    W = inputs.make_weight(wl, "fc", No=64)                  # fewer rows keep the from-scratch twin quick
+    X = inputs.make_calibration(wl, "fc")
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 1.0 / math.sqrt(X.shape[0]))
+    theta0, _ = orc.global_naive_shuffle(orc.channel_mean_metric(W, s))
+    a, ia = orc.local_block_shuffle(W, s, theta0, block=64, incremental=True)
+    b, ib = orc.local_block_shuffle(W, s, theta0, block=64, incremental=False)
+    assert np.array_equal(a, b)
+    assert np.array_equal(ia.swaps_per_block, ib.swaps_per_block)
+    assert ia.swaps_total > 0
+
+
+# ------------------------------------------------------------------------------------------ O6 select + compress
+def test_select_two_of_four_legal_nibbles_bit_copies_and_bruteforce():
+    W, X = rand_layer(50, 32, 64, 120)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.7)
+    theta = np.random.default_rng(51).permutation(64).astype(np.int32)
+    vals, meta, near = orc.select_compress(W, s, theta)
+    assert vals.shape == (32, 32) and meta.shape == (32, 8) and vals.dtype == np.float16
+    assert vals.nbytes + meta.nbytes == W.nbytes * 9 // 16     # 9/16 of dense: 43.75 % saving per layer
+    nibs = np.concatenate([(meta & 0xF).ravel(), (meta >> 4).ravel()])
+    assert set(np.unique(nibs).tolist()) <= set(orc.LEGAL_NIBBLES)
+    idx0, idx1 = orc.unpack_meta(meta)
+    assert np.all(idx0 < idx1)
+    Wp = W[:, theta]
+    dense = orc.decompress_permuted(vals, meta)
+    kept = np.zeros_like(Wp, dtype=bool).reshape(32, 16, 4)
+    np.put_along_axis(kept, idx0[:, :, None], True, axis=2)
+    np.put_along_axis(kept, idx1[:, :, None], True, axis=2)
+    kept = kept.reshape(32, 64)
+    assert np.all(kept.reshape(32, 16, 4).sum(axis=2) == 2)
+    assert np.array_equal(dense.view(np.uint16)[kept], Wp.view(np.uint16)[kept])      # bit copies
+    assert np.all(dense[~kept] == 0)
+    # brute force over the C(4,2) = 6 masks of every group: the kept pair maximises retained metric
+    xi = orc.metric(W, s)[:, theta].reshape(32, 16, 4)
+    for j in range(32):
+        for g in range(16):
+            best = max(itertools.combinations(range(4), 2), key=lambda p: (xi[j, g, p[0]] + xi[j, g, p[1]], ))
+            got = (idx0[j, g], idx1[j, g])
+            assert abs((xi[j, g, got[0]] + xi[j, g, got[1]]) - (xi[j, g, best[0]] + xi[j, g, best[1]])) < 1e-15
+    # decompress to original order is the inverse scatter
+    full = orc.decompress(vals, meta, theta)
+    assert np.array_equal(full[:, theta], dense)
+    assert not near.any() or near.dtype == bool
+
+
+def test_select_tie_break_lower_position():
+    W = np.array([[1, 1, 1, 1, 2, 1, 2, 1]], dtype=np.float16)
+    s = np.ones(8)
+    vals, meta, near = orc.select_compress(W, s, np.arange(8))
+    assert meta[0, 0] == (0x4 | (0x8 << 4))     # group 0: positions 0,1; group 1: positions 0,2
+    assert near[0, 0] and not near[0, 1]
+
+
+# ------------------------------------------------------------------------------------------ O7 product
+def test_product_invariances_and_special_cases():
+    W, X = rand_layer(60, 24, 32, 90)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.4)
+    theta = np.random.default_rng(61).permutation(32).astype(np.int32)
+    vals, meta, _ = orc.select_compress(W, s, theta)
+    Xg = np.random.default_rng(62).standard_normal((7, 32)).astype(np.float16)
+    Y = orc.product(Xg, vals, meta, theta)
+    # un-permuting the weight reproduces the product with the un-permuted input
+    Wsd = orc.decompress(vals, meta, theta).astype(np.float64)
+    assert np.allclose(Y, Xg.astype(np.float64) @ Wsd.T, rtol=1e-13, atol=1e-13)
+    # definition, entry by entry, with python loops
+    idx0, idx1 = orc.unpack_meta(meta)
+    for t, j in [(0, 0), (3, 11), (6, 23)]:
+        acc = 0.0
+        for g in range(8):
+            acc += float(vals[j, 2 * g]) * float(Xg[t, theta[4 * g + idx0[j, g]]])
+            acc += float(vals[j, 2 * g + 1]) * float(Xg[t, theta[4 * g + idx1[j, g]]])
+        assert abs(acc - Y[t, j]) < 1e-12
+    # unit rows read back rows of the un-permuted pruned weight exactly
+    E = np.eye(32, dtype=np.float16)
+    assert np.array_equal(orc.product(E, vals, meta, theta), Wsd.T)
+    # linearity in X
+    assert np.allclose(orc.product(Xg * np.float16(2), vals, meta, theta), 2 * Y, rtol=1e-15)
+    # sampled entries equal the full product
+    rows, cols = np.array([1, 5]), np.array([0, 7, 23])
+    assert np.array_equal(orc.product_entries(Xg, vals, meta, theta, rows, cols), Y[np.ix_(rows, cols)])
+
+
+def test_all_keep_permutation_invariance():
+    # with nothing pruned, X[:, theta] . W[:, theta]^T = X . W^T for any theta
+    g = np.random.default_rng(70)
+    W = g.standard_normal((5, 16)).astype(np.float16)
+    X = g.standard_normal((3, 16)).astype(np.float16)
+    theta = g.permutation(16)
+    lhs = X[:, theta].astype(np.float64) @ W[:, theta].astype(np.float64).T
+    assert np.allclose(lhs, X.astype(np.float64) @ W.astype(np.float64).T, rtol=1e-13, atol=1e-13)
+
+
+# ------------------------------------------------------------------------------------------ whole producer
+def test_metric_prune_config0_end_to_end_properties():
+    wl = inputs.WORKLOADS[0]
+    W = inputs.make_weight(wl, "fc", No=128)
+    X = inputs.make_calibration(wl, "fc")
+    r = orc.metric_prune(W, X, alpha=1.0 / math.sqrt(X.shape[0]))
+    assert sorted(r.theta.tolist()) == list(range(512))
+    assert r.obj_after_lbs >= r.obj_after_gns
+    assert abs(r.obj_after_lbs - naive_objective(W, r.score, r.theta)) <= 1e-12 * r.obj_after_lbs
+    out = inputs.outlier_channels(wl, "fc")
+    assert np.all(r.norm[out] > 5 * np.median(r.norm))           # the planted outlier channels stand out
+    assert np.all(r.entropy <= math.log(100) + 1e-12)
+    # retained metric of the final mask equals the objective
+    kept = orc.decompress_permuted(np.ones_like(r.vals), r.meta) != 0
+    xi = orc.metric(W, r.score)[:, r.theta]
+    assert abs(xi[kept].sum() - r.obj_after_lbs) <= 1e-11 * r.obj_after_lbs
