@@ -1,0 +1,180 @@
+/*
+ * esparse.h -- C ABI of the E-Sparse hot path for NVIDIA B200 (sm_100a).
+ *
+ * Two operations, as the paper states the problem:
+ *
+ *   esp_metric_prune   calibration activations + a layer's weight  ->  channel permutation,
+ *                      2:4-pruned weight in compressed form (kept values + 2-bit positions).
+ *                      Sections "Information Richness - Entropy" (Eq. 1-3), "Information Reorder -
+ *                      Channel Shuffle" (Eq. 5, Algorithm 1) and step (1) of "Efficient Sparse-GEMM
+ *                      Implementation".
+ *   esp_spgemm         the pruned layer's forward product  Y = X . P . W_s^T  on the sparse tensor
+ *                      cores ("Efficient Sparse-GEMM Implementation", Table 5).
+ *
+ * Conventions
+ *   - All tensor pointers are DEVICE pointers unless the comment says "host".  The caller owns every
+ *     buffer, including workspaces; the library allocates no device memory and keeps no state besides a
+ *     per-process cache of device properties.
+ *   - Everything is stream-ordered on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream).  Nothing synchronises unless stated.
+ *   - Inputs are never written.  Errors are return codes; argument errors are detected on the host
+ *     before anything is launched.  No call traps, aborts or throws.
+ *   - Notation: W is [No, C] row-major fp16 (No output features, C input channels); Xcal is [T, C]
+ *     fp16 calibration activations; perm[p] = original channel placed at permuted position p.
+ */
+#ifndef ESPARSE_H_
+#define ESPARSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ESP_OK = 0,
+    ESP_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, bad enum, bad struct_size        */
+    ESP_ERR_SHAPE = 2,         /* non-positive sizes, C % 8 != 0, leading dimension too small         */
+    ESP_ERR_ALIGNMENT = 3,     /* a base pointer or leading dimension is not 16-byte aligned          */
+    ESP_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than the *_workspace_bytes() answer       */
+    ESP_ERR_UNSUPPORTED = 5,   /* pattern other than 2:4, bins > 1024, device is not sm_100           */
+    ESP_ERR_CUDA = 6,          /* a CUDA runtime call or a launch failed                              */
+    ESP_ERR_TIMEOUT = 7        /* a bounded in-kernel wait gave up (reported by esp_last_device_status) */
+} esp_status_t;
+
+/* Static string for a status code (never NULL). */
+const char *esp_status_string(esp_status_t status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int esp_version(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * Pruning: metric, shuffle, 2:4 selection, compression.
+ * ---------------------------------------------------------------------------------------------- */
+
+typedef struct {
+    size_t struct_size;          /* = sizeof(esp_prune_opts)                                         */
+    double alpha;                /* weight of the norm in Eq. 3; the paper gives no value             */
+    int bins;                    /* K of Eq. 1 (paper: 100); 2..1024                                  */
+    int n_keep, m_group;         /* N:M pattern; only 2:4 is implemented on the GPU                   */
+    int lbs_block;               /* m of the local block shuffle (paper: 256); multiple of 4, <= 256  */
+    int lbs_max_swaps;           /* cap on swaps per block; 0 = until no swap improves (Algorithm 1)  */
+    int use_entropy;             /* 0 drops IR_c from the score (norm-only baseline of Table 4)       */
+    int use_norm;                /* 0 drops alpha * AM_c                                              */
+    int use_gns;                 /* 0 skips the global naive shuffle (identity start order)           */
+    int use_lbs;                 /* 0 skips the local block shuffle                                   */
+    const double *score_override;/* optional device f64[C]: use these s_c instead of computing them   */
+} esp_prune_opts;
+
+typedef struct {
+    size_t struct_size;          /* = sizeof(esp_prune_stats)                                         */
+    long long near_tie_groups;   /* groups whose 2nd and 3rd metric differ by < 1e-6 relative         */
+    long long lbs_swaps_total;   /* swaps applied by the local block shuffle                          */
+    double obj_after_gns;        /* Eq. 5 objective under the order after the global shuffle          */
+    double obj_after_lbs;        /* Eq. 5 objective under the final order                             */
+} esp_prune_stats;
+
+/* Fills *opts with the paper's settings (bins 100, 2:4, block 256, everything on, alpha = 1). */
+void esp_prune_opts_default(esp_prune_opts *opts);
+
+/* Bytes of device workspace esp_metric_prune needs for these sizes (0 on bad arguments). */
+size_t esp_metric_prune_workspace_bytes(int No, int C, int T, const esp_prune_opts *opts);
+
+/*
+ * Bytes of the tensor-core-ready copy of a compressed [No, C] weight.  Layout (opaque to callers):
+ * tiles of 128 features x 128 permuted channels, each 18432 bytes = 16384 bytes of kept fp16 values in
+ * the 128-byte-swizzled shared-memory image the MMA reads + 2048 bytes of position metadata in the
+ * order the tensor-memory copy expects.  No and C are padded up to multiples of 128 with zeros.
+ */
+size_t esp_packed_bytes(int No, int C);
+
+/*
+ * The whole producer (Eq. 1-3, global + local shuffle, 2-of-4 selection, compression).
+ *
+ *   W      [No, C] fp16, leading dimension ldw (elements, >= C, multiple of 8)
+ *   Xcal   [T, C]  fp16, leading dimension ldx (elements, >= C, multiple of 8); may be NULL when
+ *          opts->score_override is given
+ *   vals   out, fp16 [No, C/2]: kept weights, bit copies of W, two per group in position order
+ *   meta   out, u8 [No, C/8]: per group a nibble idx0 | idx1 << 2 (idx0 < idx1 = kept positions 0..3);
+ *          byte g/2 holds group g in its low (g even) or high (g odd) nibble
+ *   perm   out, int32 [C]
+ *   packed out, optional (NULL to skip): esp_packed_bytes(No, C) bytes, what esp_spgemm consumes
+ *   chan_norm / chan_entropy / chan_score  out, optional device f64[C]: AM_c, IR_c, s_c
+ *   stats  out, optional HOST struct; when non-NULL the call synchronises the stream once
+ *
+ * C must be a multiple of 8.  Returns ESP_OK or an error code; on error nothing was launched unless
+ * the code is ESP_ERR_CUDA.
+ */
+esp_status_t esp_metric_prune(const void *W, int No, int C, long ldw,
+                              const void *Xcal, int T, long ldx,
+                              const esp_prune_opts *opts,
+                              void *vals, void *meta, int32_t *perm, void *packed,
+                              double *chan_norm, double *chan_entropy, double *chan_score,
+                              esp_prune_stats *stats,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Re-tiles (vals, meta) as written by esp_metric_prune into the packed form (step (1) of "Efficient
+ * Sparse-GEMM Implementation": the compressed format the GEMM reads).  Same shapes as above.
+ */
+esp_status_t esp_pack(const void *vals, const void *meta, int No, int C, void *packed, void *cuda_stream);
+
+/*
+ * Inverse of the compression, for checking: dense fp16 [No, C] (leading dimension ldw) in ORIGINAL
+ * channel order with zeros where pruned.  perm NULL = identity.
+ */
+esp_status_t esp_decompress(const void *vals, const void *meta, const int32_t *perm, int No, int C,
+                            void *W_out, long ldw, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Sparse GEMM.
+ * ---------------------------------------------------------------------------------------------- */
+
+enum { ESP_X_TOKEN_MAJOR = 0,    /* X[t, c] at X + t * ldx + c  (tokens are rows)                      */
+       ESP_X_CHANNEL_MAJOR = 1 };/* X[t, c] at X + c * ldx + t  (channels are rows: the activation
+                                    handed over transposed)                                           */
+enum { ESP_OUT_F16 = 0, ESP_OUT_F32 = 1 };
+enum { ESP_KERNEL_AUTO = 0, ESP_KERNEL_GATHER = 1, ESP_KERNEL_TMA = 2 };
+
+typedef struct {
+    size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
+    int x_layout;                /* ESP_X_*                                                           */
+    int out_dtype;               /* ESP_OUT_*: type of Y                                              */
+    int split_k;                 /* K-slices reduced inside a thread-block cluster; 0 = choose, 1..8  */
+    int force_kernel;            /* ESP_KERNEL_*                                                      */
+    int token_tile;              /* tokens per CTA tile (16..256, multiple of 16); 0 = choose         */
+} esp_gemm_opts;
+
+void esp_gemm_opts_default(esp_gemm_opts *opts);
+
+/* Bytes of device workspace esp_spgemm needs (may be 0; then workspace may be NULL). */
+size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts);
+
+/*
+ * Y[t, j] = sum over kept weights of row j:  w * X[t, perm[position of w]]   (fp32 accumulation)
+ *
+ *   X       fp16, M tokens x K channels in the layout opts->x_layout names, leading dimension ldx
+ *           (elements; multiple of 8)
+ *   packed  esp_packed_bytes(N, K) bytes from esp_metric_prune / esp_pack
+ *   perm    int32 [K] or NULL for the identity; fused into the X-tile load, X is never copied
+ *   Y       out, [M, N] row-major (Y[t, j] at Y + t * ldy + j), fp16 or fp32 per opts->out_dtype
+ *
+ * The result does not depend on scheduling: K-slices are summed in slice order.
+ */
+esp_status_t esp_spgemm(const void *X, int M, int K, long ldx,
+                        const void *packed, const int32_t *perm, int N,
+                        void *Y, long ldy, const esp_gemm_opts *opts,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Reads and clears the device-side status word of the current device (synchronises the device).
+ * Kernels bound every wait on a barrier; a wait that gives up records ESP_ERR_TIMEOUT here and the
+ * kernel exits cleanly.  Returns ESP_OK if no kernel reported anything.
+ */
+esp_status_t esp_last_device_status(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESPARSE_H_ */

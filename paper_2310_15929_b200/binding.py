@@ -1,0 +1,186 @@
+"""ctypes binding of libesparse.so: same names as include/esparse.h, argument marshalling only.
+
+PyTorch supplies device memory and streams; every step of the path runs in the library's kernels.
+There is no fallback: if the shared library is missing the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, c_char_p, c_double, c_int, c_long, c_longlong, c_size_t, c_void_p
+
+from .build import LIB_PATH
+
+ESP_OK = 0
+ESP_ERR_INVALID_ARG, ESP_ERR_SHAPE, ESP_ERR_ALIGNMENT, ESP_ERR_WORKSPACE = 1, 2, 3, 4
+ESP_ERR_UNSUPPORTED, ESP_ERR_CUDA, ESP_ERR_TIMEOUT = 5, 6, 7
+ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
+ESP_OUT_F16, ESP_OUT_F32 = 0, 1
+ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA = 0, 1, 2
+
+
+class esp_prune_opts(ctypes.Structure):
+    _fields_ = [("struct_size", c_size_t), ("alpha", c_double), ("bins", c_int), ("n_keep", c_int),
+                ("m_group", c_int), ("lbs_block", c_int), ("lbs_max_swaps", c_int), ("use_entropy", c_int),
+                ("use_norm", c_int), ("use_gns", c_int), ("use_lbs", c_int), ("score_override", c_void_p)]
+
+
+class esp_prune_stats(ctypes.Structure):
+    _fields_ = [("struct_size", c_size_t), ("near_tie_groups", c_longlong), ("lbs_swaps_total", c_longlong),
+                ("obj_after_gns", c_double), ("obj_after_lbs", c_double)]
+
+
+class esp_gemm_opts(ctypes.Structure):
+    _fields_ = [("struct_size", c_size_t), ("x_layout", c_int), ("out_dtype", c_int), ("split_k", c_int),
+                ("force_kernel", c_int), ("token_tile", c_int)]
+
+
+class EsparseError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {esp_status_string(status)} (status {int(status)})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2310_15929_b200.build` "
+                      "(there is no CPU or PyTorch fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_gemm_opts_default",
+           "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
+           "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status")
+
+_lib.esp_status_string.restype = c_char_p
+_lib.esp_status_string.argtypes = [c_int]
+_lib.esp_version.restype = c_int
+_lib.esp_prune_opts_default.argtypes = [POINTER(esp_prune_opts)]
+_lib.esp_gemm_opts_default.argtypes = [POINTER(esp_gemm_opts)]
+_lib.esp_metric_prune_workspace_bytes.restype = c_size_t
+_lib.esp_metric_prune_workspace_bytes.argtypes = [c_int, c_int, c_int, POINTER(esp_prune_opts)]
+_lib.esp_packed_bytes.restype = c_size_t
+_lib.esp_packed_bytes.argtypes = [c_int, c_int]
+_lib.esp_metric_prune.restype = c_int
+_lib.esp_metric_prune.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_int, c_long, POINTER(esp_prune_opts),
+                                  c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                  POINTER(esp_prune_stats), c_void_p, c_size_t, c_void_p]
+_lib.esp_pack.restype = c_int
+_lib.esp_pack.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p]
+_lib.esp_decompress.restype = c_int
+_lib.esp_decompress.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_long, c_void_p]
+_lib.esp_spgemm_workspace_bytes.restype = c_size_t
+_lib.esp_spgemm_workspace_bytes.argtypes = [c_int, c_int, c_int, POINTER(esp_gemm_opts)]
+_lib.esp_spgemm.restype = c_int
+_lib.esp_spgemm.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
+                            POINTER(esp_gemm_opts), c_void_p, c_size_t, c_void_p]
+_lib.esp_last_device_status.restype = c_int
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / raw int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def esp_status_string(status: int) -> str:
+    return _lib.esp_status_string(int(status)).decode()
+
+
+def esp_version() -> int:
+    return int(_lib.esp_version())
+
+
+def esp_prune_opts_default() -> esp_prune_opts:
+    o = esp_prune_opts()
+    _lib.esp_prune_opts_default(ctypes.byref(o))
+    return o
+
+
+def esp_gemm_opts_default() -> esp_gemm_opts:
+    o = esp_gemm_opts()
+    _lib.esp_gemm_opts_default(ctypes.byref(o))
+    return o
+
+
+def esp_metric_prune_workspace_bytes(No: int, C: int, T: int, opts: esp_prune_opts) -> int:
+    return int(_lib.esp_metric_prune_workspace_bytes(No, C, T, ctypes.byref(opts)))
+
+
+def esp_packed_bytes(No: int, C: int) -> int:
+    return int(_lib.esp_packed_bytes(No, C))
+
+
+def esp_metric_prune_raw(W, No, C, ldw, Xcal, T, ldx, opts, vals, meta, perm, packed, chan_norm, chan_entropy,
+                         chan_score, stats, workspace, workspace_bytes, stream) -> int:
+    """The C call with raw addresses; returns the status code without raising (used by error-path tests)."""
+    return int(_lib.esp_metric_prune(_ptr(W), No, C, ldw, _ptr(Xcal), T, ldx,
+                                     ctypes.byref(opts) if opts is not None else None,
+                                     _ptr(vals), _ptr(meta), _ptr(perm), _ptr(packed), _ptr(chan_norm),
+                                     _ptr(chan_entropy), _ptr(chan_score),
+                                     ctypes.byref(stats) if stats is not None else None,
+                                     _ptr(workspace), workspace_bytes, stream))
+
+
+def esp_metric_prune(W, Xcal, opts, vals, meta, perm, packed=None, chan_norm=None, chan_entropy=None,
+                     chan_score=None, stats=None, workspace=None, stream=None):
+    """W [No,C] f16, Xcal [T,C] f16 (or None with opts.score_override) -> vals, meta, perm (, packed)."""
+    No, C = W.shape
+    T = 0 if Xcal is None else Xcal.shape[0]
+    ldx = C if Xcal is None else Xcal.stride(0)
+    if stats is not None:
+        stats.struct_size = ctypes.sizeof(esp_prune_stats)
+    st = esp_metric_prune_raw(W, No, C, W.stride(0), Xcal, T, ldx, opts, vals, meta, perm, packed, chan_norm,
+                              chan_entropy, chan_score, stats, workspace,
+                              0 if workspace is None else workspace.numel() * workspace.element_size(),
+                              _stream(stream))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_metric_prune")
+
+
+def esp_pack(vals, meta, No, C, packed, stream=None):
+    st = int(_lib.esp_pack(_ptr(vals), _ptr(meta), No, C, _ptr(packed), _stream(stream)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_pack")
+
+
+def esp_decompress(vals, meta, perm, No, C, W_out, stream=None):
+    st = int(_lib.esp_decompress(_ptr(vals), _ptr(meta), _ptr(perm), No, C, _ptr(W_out), W_out.stride(0),
+                                 _stream(stream)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_decompress")
+
+
+def esp_spgemm_workspace_bytes(M: int, N: int, K: int, opts: esp_gemm_opts) -> int:
+    return int(_lib.esp_spgemm_workspace_bytes(M, N, K, ctypes.byref(opts)))
+
+
+def esp_spgemm_raw(X, M, K, ldx, packed, perm, N, Y, ldy, opts, workspace, workspace_bytes, stream) -> int:
+    return int(_lib.esp_spgemm(_ptr(X), M, K, ldx, _ptr(packed), _ptr(perm), N, _ptr(Y), ldy,
+                               ctypes.byref(opts) if opts is not None else None, _ptr(workspace), workspace_bytes,
+                               stream))
+
+
+def esp_spgemm(X, packed, perm, Y, opts, workspace=None, stream=None):
+    """Y [M,N] = X . P . W_s^T.  X is [M,K] (token-major) or [K,M] (channel-major) per opts.x_layout."""
+    M, N = Y.shape
+    if opts.x_layout == ESP_X_CHANNEL_MAJOR:
+        K = X.shape[0]
+    else:
+        K = X.shape[1]
+    st = esp_spgemm_raw(X, M, K, X.stride(0), packed, perm, N, Y, Y.stride(0), opts, workspace,
+                        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_spgemm")
+
+
+def esp_last_device_status() -> int:
+    return int(_lib.esp_last_device_status())

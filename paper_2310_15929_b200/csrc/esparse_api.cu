@@ -1,0 +1,182 @@
+// C ABI of the esparse library: argument validation on the host, then stream-ordered launches.
+#include "esp_common.cuh"
+
+#include <mutex>
+
+namespace esp {
+
+esp_status_t device_info(DeviceInfo *out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = -1;
+    ESP_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ESP_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev].device != dev) {
+        DeviceInfo d;
+        d.device = dev;
+        ESP_CUDA_OK(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        ESP_CUDA_OK(cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+        ESP_CUDA_OK(cudaDeviceGetAttribute(&d.cc_minor, cudaDevAttrComputeCapabilityMinor, dev));
+        ESP_CUDA_OK(cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        cache[dev] = d;
+    }
+    *out = cache[dev];
+    return ESP_OK;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static esp_status_t check_prune_opts(const esp_prune_opts *o) {
+    if (!o || o->struct_size != sizeof(esp_prune_opts)) return ESP_ERR_INVALID_ARG;
+    if (o->n_keep != 2 || o->m_group != 4) return ESP_ERR_UNSUPPORTED;
+    if (o->bins < 2 || o->bins > 512) return ESP_ERR_UNSUPPORTED;
+    if (o->lbs_block < 4 || o->lbs_block > 256 || o->lbs_block % 4 != 0) return ESP_ERR_INVALID_ARG;
+    if (o->lbs_max_swaps < 0) return ESP_ERR_INVALID_ARG;
+    return ESP_OK;
+}
+
+static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
+    if (!o || o->struct_size != sizeof(esp_gemm_opts)) return ESP_ERR_INVALID_ARG;
+    if (o->x_layout != ESP_X_TOKEN_MAJOR && o->x_layout != ESP_X_CHANNEL_MAJOR) return ESP_ERR_INVALID_ARG;
+    if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
+    if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
+    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_TMA) return ESP_ERR_INVALID_ARG;
+    if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
+    return ESP_OK;
+}
+
+}  // namespace esp
+
+using namespace esp;
+
+extern "C" {
+
+const char *esp_status_string(esp_status_t status) {
+    switch (status) {
+        case ESP_OK: return "ok";
+        case ESP_ERR_INVALID_ARG: return "invalid argument";
+        case ESP_ERR_SHAPE: return "bad shape or leading dimension";
+        case ESP_ERR_ALIGNMENT: return "pointer or leading dimension not 16-byte aligned";
+        case ESP_ERR_WORKSPACE: return "workspace missing or too small";
+        case ESP_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case ESP_ERR_CUDA: return "CUDA runtime error";
+        case ESP_ERR_TIMEOUT: return "a bounded in-kernel wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int esp_version(void) { return 100; }
+
+void esp_prune_opts_default(esp_prune_opts *o) {
+    if (!o) return;
+    o->struct_size = sizeof(esp_prune_opts);
+    o->alpha = 1.0;
+    o->bins = 100;
+    o->n_keep = 2;
+    o->m_group = 4;
+    o->lbs_block = 256;
+    o->lbs_max_swaps = 0;
+    o->use_entropy = 1;
+    o->use_norm = 1;
+    o->use_gns = 1;
+    o->use_lbs = 1;
+    o->score_override = nullptr;
+}
+
+void esp_gemm_opts_default(esp_gemm_opts *o) {
+    if (!o) return;
+    o->struct_size = sizeof(esp_gemm_opts);
+    o->x_layout = ESP_X_TOKEN_MAJOR;
+    o->out_dtype = ESP_OUT_F16;
+    o->split_k = 0;
+    o->force_kernel = ESP_KERNEL_AUTO;
+    o->token_tile = 0;
+}
+
+size_t esp_metric_prune_workspace_bytes(int No, int C, int T, const esp_prune_opts *opts) {
+    if (No <= 0 || C <= 0 || T < 0 || C % 8 != 0 || check_prune_opts(opts) != ESP_OK) return 0;
+    return carve_prune_workspace(nullptr, No, C, T, *opts).total_bytes;
+}
+
+size_t esp_packed_bytes(int No, int C) {
+    if (No <= 0 || C <= 0) return 0;
+    return (size_t)ceil_div(No, kTileFeat) * (size_t)ceil_div(C, kTileK) * (size_t)kTileBytes;
+}
+
+esp_status_t esp_metric_prune(const void *W, int No, int C, long ldw, const void *Xcal, int T, long ldx,
+                              const esp_prune_opts *opts, void *vals, void *meta, int32_t *perm, void *packed,
+                              double *chan_norm, double *chan_entropy, double *chan_score, esp_prune_stats *stats,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    esp_status_t st = check_prune_opts(opts);
+    if (st != ESP_OK) return st;
+    if (!W || !vals || !meta || !perm) return ESP_ERR_INVALID_ARG;
+    if (!Xcal && !opts->score_override) return ESP_ERR_INVALID_ARG;
+    if (stats && stats->struct_size != sizeof(esp_prune_stats)) return ESP_ERR_INVALID_ARG;
+    if (No <= 0 || C <= 0 || C % 8 != 0 || ldw < C) return ESP_ERR_SHAPE;
+    if (Xcal && (T <= 0 || ldx < C)) return ESP_ERR_SHAPE;
+    if (ldw % 8 != 0 || (Xcal && ldx % 8 != 0)) return ESP_ERR_ALIGNMENT;
+    if (!aligned16(W) || !aligned16(Xcal) || !aligned16(vals) || !aligned16(meta) || !aligned16(perm) ||
+        !aligned16(packed) || !aligned16(workspace))
+        return ESP_ERR_ALIGNMENT;
+    PruneWorkspace w = carve_prune_workspace(workspace, No, C, Xcal ? T : 0, *opts);
+    if (!workspace || workspace_bytes < w.total_bytes) return ESP_ERR_WORKSPACE;
+    DeviceInfo di;
+    st = device_info(&di);
+    if (st != ESP_OK) return st;
+    if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
+    return launch_prune((const __half *)W, No, C, ldw, (const __half *)Xcal, Xcal ? T : 0, ldx, *opts, (__half *)vals,
+                        (uint8_t *)meta, perm, packed, chan_norm, chan_entropy, chan_score, stats, w,
+                        (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_pack(const void *vals, const void *meta, int No, int C, void *packed, void *cuda_stream) {
+    if (!vals || !meta || !packed) return ESP_ERR_INVALID_ARG;
+    if (No <= 0 || C <= 0 || C % 8 != 0) return ESP_ERR_SHAPE;
+    if (!aligned16(vals) || !aligned16(meta) || !aligned16(packed)) return ESP_ERR_ALIGNMENT;
+    return launch_pack((const __half *)vals, (const uint8_t *)meta, No, C, packed, (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_decompress(const void *vals, const void *meta, const int32_t *perm, int No, int C, void *W_out,
+                            long ldw, void *cuda_stream) {
+    if (!vals || !meta || !W_out) return ESP_ERR_INVALID_ARG;
+    if (No <= 0 || C <= 0 || C % 8 != 0 || ldw < C) return ESP_ERR_SHAPE;
+    return launch_decompress((const __half *)vals, (const uint8_t *)meta, perm, No, C, (__half *)W_out, ldw,
+                             (cudaStream_t)cuda_stream);
+}
+
+size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts) {
+    (void)M; (void)N; (void)K; (void)opts;
+    return 0;   // K-slices are reduced through distributed shared memory inside a cluster: no global scratch
+}
+
+esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
+                        void *Y, long ldy, const esp_gemm_opts *opts, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream) {
+    esp_status_t st = check_gemm_opts(opts);
+    if (st != ESP_OK) return st;
+    if (!X || !packed || !Y) return ESP_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 8 != 0 || ldy < N) return ESP_ERR_SHAPE;
+    if (opts->x_layout == ESP_X_TOKEN_MAJOR ? (ldx < K) : (ldx < M)) return ESP_ERR_SHAPE;
+    if (ldx % 8 != 0) return ESP_ERR_ALIGNMENT;
+    if (!aligned16(X) || !aligned16(packed) || !aligned16(Y) || !aligned16(perm)) return ESP_ERR_ALIGNMENT;
+    DeviceInfo di;
+    st = device_info(&di);
+    if (st != ESP_OK) return st;
+    if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
+    GemmPlan plan;
+    st = plan_gemm(M, N, K, *opts, &plan);
+    if (st != ESP_OK) return st;
+    return launch_spgemm((const __half *)X, M, K, ldx, packed, perm, N, Y, ldy, *opts, plan, workspace,
+                         workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_last_device_status(void) {
+    int h = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return ESP_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return ESP_ERR_CUDA;
+    if (h != 0 && cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return ESP_ERR_CUDA;
+    return (esp_status_t)h;
+}
+
+}  // extern "C"

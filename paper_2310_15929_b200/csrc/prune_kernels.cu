@@ -1,0 +1,738 @@
+// Producer side of the E-Sparse hot path: channel statistics (Eq. 1, Eq. 2), score (Eq. 3), global
+// naive shuffle, local block shuffle (Algorithm 1, Eq. 5), 2-of-4 selection and compression.
+//
+// All of these stream fp16 matrices once or twice; they are HBM-bound or (block shuffle) bound by plain
+// fp64 compares.  Every quantity that feeds a discrete decision is fp64 with explicit round-to-nearest
+// multiplies/adds (no FMA contraction), and every sum over rows of |W| is taken exactly in 64-bit
+// integers of 2^-24, so results do not depend on the order in which threads visit rows.
+#include "esp_common.cuh"
+
+#include <math.h>
+
+namespace esp {
+
+namespace {
+
+constexpr int kLbsMax = 256;       // widest local-shuffle block
+constexpr int kLbsGroups = kLbsMax / 4;
+
+__device__ __forceinline__ double half_bits_abs_to_double(uint16_t h) {
+    return (double)__half2float(__ushort_as_half((unsigned short)(h & 0x7FFFu)));
+}
+
+// |h| as an integer multiple of 2^-24 (exact for every finite fp16).
+__device__ __forceinline__ long long half_bits_abs_fixed(uint16_t h) {
+    int e = (h >> 10) & 31;
+    long long m = h & 1023;
+    return e == 0 ? m : ((1024 + m) << (e - 1));
+}
+
+// --------------------------------------------------------------------------------------------------
+// K1: per-channel sum of squares (fp64), min and max over a slice of tokens.   Eq. 2 / range of Eq. 1.
+// grid (ceil(C/256), splits), block 256 = 32 channel-vectors of 8 x 8 token lanes.
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) colstats_kernel(const __half *__restrict__ X, int T, int C, long ldx,
+                                                       int rows_per_split, double *__restrict__ part_sumsq,
+                                                       float *__restrict__ part_min, float *__restrict__ part_max) {
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int c0 = (blockIdx.x * 32 + tx) * 8;
+    const int r_begin = blockIdx.y * rows_per_split;
+    const int r_end = min(T, r_begin + rows_per_split);
+    double acc[8];
+    float mn[8], mx[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { acc[k] = 0.0; mn[k] = INFINITY; mx[k] = -INFINITY; }
+    if (c0 < C) {
+        for (int r = r_begin + ty; r < r_end; r += 8) {
+            uint4 v = __ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0));
+            const __half *h = reinterpret_cast<const __half *>(&v);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                float f = __half2float(h[k]);
+                acc[k] = __dadd_rn(acc[k], (double)(f * f));   // f*f is exact in fp32 (22-bit product)
+                mn[k] = fminf(mn[k], f);
+                mx[k] = fmaxf(mx[k], f);
+            }
+        }
+    }
+    __shared__ double s_acc[8][256 + 1];
+    __shared__ float s_mn[8][256 + 1], s_mx[8][256 + 1];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { s_acc[ty][tx * 8 + k] = acc[k]; s_mn[ty][tx * 8 + k] = mn[k]; s_mx[ty][tx * 8 + k] = mx[k]; }
+    __syncthreads();
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (c < C) {
+        double a = 0.0;
+        float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) {      // fixed order: deterministic
+            a = __dadd_rn(a, s_acc[y][threadIdx.x]);
+            lo = fminf(lo, s_mn[y][threadIdx.x]);
+            hi = fmaxf(hi, s_mx[y][threadIdx.x]);
+        }
+        part_sumsq[(long)blockIdx.y * C + c] = a;
+        part_min[(long)blockIdx.y * C + c] = lo;
+        part_max[(long)blockIdx.y * C + c] = hi;
+    }
+}
+
+__global__ void colstats_finish_kernel(int C, int splits, const double *__restrict__ part_sumsq,
+                                       const float *__restrict__ part_min, const float *__restrict__ part_max,
+                                       double *__restrict__ norm, double *__restrict__ lo, double *__restrict__ hi) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double a = 0.0;
+    float mn = INFINITY, mx = -INFINITY;
+    for (int s = 0; s < splits; ++s) {
+        a = __dadd_rn(a, part_sumsq[(long)s * C + c]);
+        mn = fminf(mn, part_min[(long)s * C + c]);
+        mx = fmaxf(mx, part_max[(long)s * C + c]);
+    }
+    norm[c] = sqrt(a);
+    lo[c] = (double)mn;
+    hi[c] = (double)mx;
+}
+
+// --------------------------------------------------------------------------------------------------
+// K2: per-channel histogram with K equal-width bins on [lo_c, hi_c] (Eq. 1's bins), exact integer counts.
+// bin = min(K-1, floor((x - lo) * K / (hi - lo))) in fp64: the numerator is exact and the quotient is
+// correctly rounded, which yields the exact bin for fp16 data.
+// grid (ceil(C/64), splits), block 256 = 8 channel-vectors of 8 x 32 token lanes; counters in shared memory.
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) histogram_kernel(const __half *__restrict__ X, int T, int C, long ldx,
+                                                        int rows_per_split, int bins, const double *__restrict__ lo,
+                                                        const double *__restrict__ hi, unsigned int *__restrict__ counts) {
+    extern __shared__ unsigned int s_cnt[];   // [64][bins]
+    for (int i = threadIdx.x; i < 64 * bins; i += 256) s_cnt[i] = 0;
+    __syncthreads();
+    const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;
+    const int cl = tx * 8;
+    const int c0 = blockIdx.x * 64 + cl;
+    const int r_begin = blockIdx.y * rows_per_split;
+    const int r_end = min(T, r_begin + rows_per_split);
+    if (c0 < C) {
+        double l[8], scale_den[8];
+        bool flat[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            l[k] = lo[c0 + k];
+            double rng = __dsub_rn(hi[c0 + k], l[k]);
+            flat[k] = !(rng > 0.0);
+            scale_den[k] = flat[k] ? 1.0 : rng;
+        }
+        const double kb = (double)bins;
+        for (int r = r_begin + ty; r < r_end; r += 32) {
+            uint4 v = __ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0));
+            const __half *h = reinterpret_cast<const __half *>(&v);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                double x = (double)__half2float(h[k]);
+                double q = __ddiv_rn(__dmul_rn(__dsub_rn(x, l[k]), kb), scale_den[k]);
+                int b = flat[k] ? 0 : min(bins - 1, (int)floor(q));
+                atomicAdd(&s_cnt[(cl + k) * bins + b], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 64 * bins; i += 256) {
+        int c = blockIdx.x * 64 + i / bins;
+        unsigned int n = s_cnt[i];
+        if (c < C && n) atomicAdd(&counts[(long)c * bins + (i % bins)], n);
+    }
+}
+
+// IR_c = -sum_k p_k ln p_k (Eq. 1, bins in index order, empty bins skipped) and s_c = IR_c + alpha*AM_c (Eq. 3).
+__global__ void entropy_score_kernel(int C, int T, int bins, const unsigned int *__restrict__ counts,
+                                     const double *__restrict__ norm, double alpha, int use_entropy, int use_norm,
+                                     const double *__restrict__ score_override, double *__restrict__ entropy,
+                                     double *__restrict__ score) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double ir = 0.0;
+    if (counts) {
+        for (int k = 0; k < bins; ++k) {
+            unsigned int n = counts[(long)c * bins + k];
+            if (n) {
+                double p = __ddiv_rn((double)n, (double)T);
+                ir = __dsub_rn(ir, __dmul_rn(p, log(p)));
+            }
+        }
+        entropy[c] = ir;
+    }
+    double s = 0.0;
+    if (score_override) {
+        s = score_override[c];
+    } else {
+        if (use_entropy) s = __dadd_rn(s, ir);
+        if (use_norm) s = __dadd_rn(s, __dmul_rn(alpha, norm[c]));
+    }
+    score[c] = s;
+}
+
+// --------------------------------------------------------------------------------------------------
+// K3: exact column sums of |W| (units of 2^-24) -> mean of the metric per channel (for the global shuffle).
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) colabs_kernel(const __half *__restrict__ W, int No, int C, long ldw,
+                                                     int rows_per_split, unsigned long long *__restrict__ colsum) {
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int c0 = (blockIdx.x * 32 + tx) * 8;
+    const int r_begin = blockIdx.y * rows_per_split;
+    const int r_end = min(No, r_begin + rows_per_split);
+    long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (c0 < C) {
+        for (int r = r_begin + ty; r < r_end; r += 8) {
+            uint4 v = __ldg(reinterpret_cast<const uint4 *>(W + (long)r * ldw + c0));
+            const uint16_t *h = reinterpret_cast<const uint16_t *>(&v);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] += half_bits_abs_fixed(h[k]);
+        }
+    }
+    __shared__ long long s_acc[8][256 + 1];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s_acc[ty][tx * 8 + k] = acc[k];
+    __syncthreads();
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (c < C) {
+        long long a = 0;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) a += s_acc[y][threadIdx.x];
+        atomicAdd(&colsum[c], (unsigned long long)a);      // integer: order-independent
+    }
+}
+
+__global__ void mean_metric_kernel(int C, int No, const unsigned long long *__restrict__ colsum,
+                                   const double *__restrict__ score, double *__restrict__ mean) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double a = __dmul_rn(__ll2double_rn((long long)colsum[c]), 0x1p-24);
+    mean[c] = __ddiv_rn(__dmul_rn(score[c], a), (double)No);
+}
+
+// --------------------------------------------------------------------------------------------------
+// K4: global naive shuffle.  rank(c) = number of channels ahead of c in a stable descending sort of the
+// mean metric; the channel of rank r goes to group r mod G, slot r div G (neighbours in rank never share
+// a group).
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__restrict__ mean, int use_gns,
+                                                       int32_t *__restrict__ theta0) {
+    __shared__ double tile[256];
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (!use_gns) {
+        if (c < C) theta0[c] = c;
+        return;
+    }
+    const double mine = (c < C) ? mean[c] : 0.0;
+    int rank = 0;
+    for (int base = 0; base < C; base += 256) {
+        __syncthreads();
+        if (base + threadIdx.x < C) tile[threadIdx.x] = mean[base + threadIdx.x];
+        __syncthreads();
+        const int n = min(256, C - base);
+        for (int i = 0; i < n; ++i) {
+            double other = tile[i];
+            rank += (other > mine || (other == mine && base + i < c)) ? 1 : 0;
+        }
+    }
+    if (c < C) {
+        const int G = C / 4;
+        theta0[(rank % G) * 4 + rank / G] = c;
+    }
+}
+
+// --------------------------------------------------------------------------------------------------
+// K5: local block shuffle (Algorithm 1 lines 3-14).
+// Wt[c][j] = |W[j,c]| bits, channel-major and zero-padded to ldt rows, so a channel's column is contiguous.
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) abs_transpose_kernel(const __half *__restrict__ W, int No, int C, long ldw,
+                                                            uint16_t *__restrict__ Wt, long ldt) {
+    __shared__ uint16_t tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int c_base = blockIdx.x * 32, r_base = blockIdx.y * 32;
+    const uint16_t *Wb = reinterpret_cast<const uint16_t *>(W);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int r = r_base + ty + i * 8, c = c_base + tx;
+        tile[ty + i * 8][tx] = (r < No && c < C) ? (uint16_t)(Wb[(long)r * ldw + c] & 0x7FFFu) : (uint16_t)0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int c = c_base + ty + i * 8, r = r_base + tx;
+        if (c < C && r < ldt) Wt[(long)c * ldt + r] = tile[tx][ty + i * 8];
+    }
+}
+
+// Retained metric sum of one group of 4 channels over all rows (Eq. 5 restricted to the group), computed
+// by one warp.  Every lane returns the value.
+//   kept(j,k): slot k is among the 2 largest xi[j,.] = |w| * s (ties: lower slot)
+//   A_k = sum_j kept(j,k) |w_jk| exactly;  V = ((s0*a0 + s1*a1) + s2*a2) + s3*a3
+__device__ double group_value_warp(const uint16_t *__restrict__ Wt, long ldt, const double *__restrict__ score,
+                                   int c0, int c1, int c2, int c3) {
+    const int lane = threadIdx.x & 31;
+    const int ch[4] = {c0, c1, c2, c3};
+    double sc[4];
+    long long A[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) sc[k] = score[ch[k]];
+    for (long j = lane * 8; j < ldt; j += 256) {
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[k] = *reinterpret_cast<const uint4 *>(Wt + (long)ch[k] * ldt + j);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            uint16_t h[4];
+            double xi[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                h[k] = reinterpret_cast<const uint16_t *>(&v[k])[e];
+                xi[k] = __dmul_rn(half_bits_abs_to_double(h[k]), sc[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int ahead = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (q == k) continue;
+                    ahead += (xi[q] > xi[k] || (xi[q] == xi[k] && q < k)) ? 1 : 0;
+                }
+                if (ahead < 2) A[k] += half_bits_abs_fixed(h[k]);
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) A[k] += __shfl_xor_sync(0xFFFFFFFFu, A[k], off);
+    }
+    double t0 = __dmul_rn(sc[0], __dmul_rn(__ll2double_rn(A[0]), 0x1p-24));
+    double t1 = __dmul_rn(sc[1], __dmul_rn(__ll2double_rn(A[1]), 0x1p-24));
+    double t2 = __dmul_rn(sc[2], __dmul_rn(__ll2double_rn(A[2]), 0x1p-24));
+    double t3 = __dmul_rn(sc[3], __dmul_rn(__ll2double_rn(A[3]), 0x1p-24));
+    return __dadd_rn(__dadd_rn(__dadd_rn(t0, t1), t2), t3);
+}
+
+// table[b][g][slot][x] = V(group g of block b with its slot replaced by block channel x); base[G] = V(g).
+// grid (nblocks * 64), block 256 (8 warps).
+__global__ void __launch_bounds__(256) lbs_table_kernel(const uint16_t *__restrict__ Wt, long ldt,
+                                                        const double *__restrict__ score,
+                                                        const int32_t *__restrict__ theta0, int C, int lbs_block,
+                                                        double *__restrict__ table, double *__restrict__ base) {
+    const int b = blockIdx.x / kLbsGroups, g = blockIdx.x % kLbsGroups;
+    const int p0 = b * lbs_block;
+    const int m = min(lbs_block, C - p0);
+    if (g * 4 >= m) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int grp[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) grp[k] = theta0[p0 + g * 4 + k];
+    double *tb = table + ((long)b * kLbsGroups + g) * 4 * kLbsMax;
+    for (int e = warp; e < 4 * m; e += 8) {
+        const int slot = e / m, x = e % m;
+        double v = 0.0;
+        if (x / 4 != g) {
+            int ch[4] = {grp[0], grp[1], grp[2], grp[3]};
+            ch[slot] = theta0[p0 + x];
+            v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
+        }
+        if (lane == 0) tb[slot * kLbsMax + x] = v;
+    }
+    if (warp == 0) {
+        double v = group_value_warp(Wt, ldt, score, grp[0], grp[1], grp[2], grp[3]);
+        if (lane == 0) base[p0 / 4 + g] = v;
+    }
+}
+
+// One CTA per block of positions: repeat { best cross-group swap by table lookup; apply if gain > 0;
+// refresh the two touched groups }.  grid (nblocks), block 512.
+__global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restrict__ Wt, long ldt,
+                                                          const double *__restrict__ score,
+                                                          const int32_t *__restrict__ theta0, int C, int lbs_block,
+                                                          int max_swaps, double *__restrict__ table,
+                                                          double *__restrict__ base, int32_t *__restrict__ theta,
+                                                          unsigned long long *__restrict__ counters) {
+    const int b = blockIdx.x;
+    const int p0 = b * lbs_block;
+    const int m = min(lbs_block, C - p0);
+    const int G = m / 4;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    __shared__ int pos2x[kLbsMax];
+    __shared__ int chan[kLbsMax];
+    __shared__ double s_base[kLbsGroups];
+    __shared__ double red_gain[16];
+    __shared__ int red_idx[16];
+    __shared__ int decision;      // linear pair index i*256+j, or -1 to stop
+    double *tb = table + (long)b * kLbsGroups * 4 * kLbsMax;
+    if (tid < m) { pos2x[tid] = tid; chan[tid] = theta0[p0 + tid]; }
+    if (tid < G) s_base[tid] = base[p0 / 4 + tid];
+    __syncthreads();
+    int swaps = 0;
+    for (;;) {
+        double best = -INFINITY;
+        int best_e = 0x7FFFFFFF;
+        if (max_swaps <= 0 || swaps < max_swaps) {
+            for (int e = tid; e < kLbsMax * kLbsMax; e += 512) {
+                const int i = e >> 8, j = e & 255;
+                if (j <= i || j >= m || (i >> 2) == (j >> 2)) continue;
+                const int gi = i >> 2, si = i & 3, gj = j >> 2, sj = j & 3;
+                double after = __dadd_rn(tb[(gi * 4 + si) * kLbsMax + pos2x[j]], tb[(gj * 4 + sj) * kLbsMax + pos2x[i]]);
+                double gain = __dsub_rn(after, __dadd_rn(s_base[gi], s_base[gj]));
+                if (gain > best || (gain == best && e < best_e)) { best = gain; best_e = e; }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            double og = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+            int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
+            if (og > best || (og == best && oe < best_e)) { best = og; best_e = oe; }
+        }
+        if (lane == 0) { red_gain[warp] = best; red_idx[warp] = best_e; }
+        __syncthreads();
+        if (warp == 0) {
+            best = lane < 16 ? red_gain[lane] : -INFINITY;
+            best_e = lane < 16 ? red_idx[lane] : 0x7FFFFFFF;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                double og = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+                int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
+                if (og > best || (og == best && oe < best_e)) { best = og; best_e = oe; }
+            }
+            if (lane == 0) decision = (best > 0.0) ? best_e : -1;
+        }
+        __syncthreads();
+        const int d = decision;
+        if (d < 0) break;
+        const int bi = d >> 8, bj = d & 255;
+        if (tid == 0) { int t = pos2x[bi]; pos2x[bi] = pos2x[bj]; pos2x[bj] = t; }
+        ++swaps;
+        __syncthreads();
+        // refresh base and table rows of the two touched groups: 2 * (1 + 4*m) group evaluations
+        const int per_group = 1 + 4 * m;
+        for (int w = warp; w < 2 * per_group; w += 16) {
+            const int g = (w < per_group) ? (bi >> 2) : (bj >> 2);
+            const int e = (w < per_group) ? w : w - per_group;
+            int ch[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) ch[k] = chan[pos2x[g * 4 + k]];
+            if (e == 0) {
+                double v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
+                if (lane == 0) s_base[g] = v;
+            } else {
+                const int slot = (e - 1) / m, x = (e - 1) % m;
+                ch[slot] = chan[x];
+                double v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
+                if (lane == 0) tb[(g * 4 + slot) * kLbsMax + x] = v;
+            }
+        }
+        __syncthreads();
+    }
+    if (tid < m) theta[p0 + tid] = chan[pos2x[tid]];
+    if (tid < G) base[p0 / 4 + tid] = s_base[tid];
+    if (tid == 0 && swaps) atomicAdd(&counters[1], (unsigned long long)swaps);
+}
+
+// Sum of the group values in group order (Eq. 5 objective), one thread: deterministic.
+__global__ void objective_kernel(int G, const double *__restrict__ base, double *__restrict__ out) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        double t = 0.0;
+        for (int g = 0; g < G; ++g) t = __dadd_rn(t, base[g]);
+        *out = t;
+    }
+}
+
+// base[g] = V(g) under theta for every group (used when the block shuffle is off but stats are wanted).
+__global__ void __launch_bounds__(256) group_values_kernel(const uint16_t *__restrict__ Wt, long ldt,
+                                                           const double *__restrict__ score,
+                                                           const int32_t *__restrict__ theta, int G,
+                                                           double *__restrict__ base) {
+    const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (g >= G) return;
+    double v = group_value_warp(Wt, ldt, score, theta[4 * g], theta[4 * g + 1], theta[4 * g + 2], theta[4 * g + 3]);
+    if ((threadIdx.x & 31) == 0) base[g] = v;
+}
+
+// --------------------------------------------------------------------------------------------------
+// K6: 2-of-4 selection + compression.  One CTA per output row: the row is staged in shared memory, then
+// each thread handles 8 permuted positions (2 groups): 4 kept values + 1 metadata byte.
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) select_compress_kernel(const __half *__restrict__ W, int No, int C, long ldw,
+                                                              const double *__restrict__ score,
+                                                              const int32_t *__restrict__ theta,
+                                                              __half *__restrict__ vals, uint8_t *__restrict__ meta,
+                                                              unsigned long long *__restrict__ counters) {
+    extern __shared__ uint16_t s_row[];
+    const int j = blockIdx.x;
+    const uint16_t *Wr = reinterpret_cast<const uint16_t *>(W) + (long)j * ldw;
+    for (int c = threadIdx.x * 8; c < C; c += 256 * 8)
+        *reinterpret_cast<uint4 *>(s_row + c) = __ldg(reinterpret_cast<const uint4 *>(Wr + c));
+    __syncthreads();
+    unsigned int near = 0;
+    for (int u = threadIdx.x; u < C / 8; u += 256) {
+        uint16_t out[4];
+        unsigned int byte = 0;
+#pragma unroll
+        for (int gg = 0; gg < 2; ++gg) {
+            uint16_t h[4];
+            double xi[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int c = theta[u * 8 + gg * 4 + k];
+                h[k] = s_row[c];
+                xi[k] = __dmul_rn(half_bits_abs_to_double(h[k]), score[c]);
+            }
+            int kept[2], nk = 0;
+            double second = 0.0, third = 0.0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int ahead = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (q == k) continue;
+                    ahead += (xi[q] > xi[k] || (xi[q] == xi[k] && q < k)) ? 1 : 0;
+                }
+                if (ahead < 2) { if (nk < 2) kept[nk] = k; ++nk; }
+                if (ahead == 1) second = xi[k];
+                if (ahead == 2) third = xi[k];
+            }
+            if (__dsub_rn(second, third) < __dmul_rn(1e-6, second)) ++near;
+            out[gg * 2 + 0] = h[kept[0]];
+            out[gg * 2 + 1] = h[kept[1]];
+            byte |= (unsigned int)(kept[0] | (kept[1] << 2)) << (4 * gg);
+        }
+        uint2 packed;
+        packed.x = (unsigned int)out[0] | ((unsigned int)out[1] << 16);
+        packed.y = (unsigned int)out[2] | ((unsigned int)out[3] << 16);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(vals) + (long)j * (C / 2) + u * 4) = packed;
+        meta[(long)j * (C / 8) + u] = (uint8_t)byte;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) near += __shfl_xor_sync(0xFFFFFFFFu, near, off);
+    if ((threadIdx.x & 31) == 0 && near) atomicAdd(&counters[0], (unsigned long long)near);
+}
+
+// --------------------------------------------------------------------------------------------------
+// K7: re-tile (vals, meta) into the layout the sparse MMA reads.
+// Per (feature tile ft, channel tile kt) 18432 contiguous bytes:
+//   [0, 16384)      128 rows x 128 bytes of kept values, 16-byte chunk q of row r stored at chunk q ^ (r & 7)
+//                   (the 128-byte swizzle of a K-major shared-memory operand)
+//   [16384, 18432)  128 lanes x 4 words; lane l, word c: low half = metadata of row (l&7) + 16*(l>>4), high half =
+//                   that row + 8, for channels 32c + 16*((l>>3)&1) .. +16 of the tile (the order in which the
+//                   tensor-memory copy lays 16 bytes per lane next to the accumulator lanes)
+// --------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_kernel(const __half *__restrict__ vals, const uint8_t *__restrict__ meta,
+                                                   int No, int C, uint8_t *__restrict__ packed, int k_tiles) {
+    const int kt = blockIdx.x, ft = blockIdx.y;
+    uint8_t *tile = packed + ((long)ft * k_tiles + kt) * kTileBytes;
+    const uint16_t *v16 = reinterpret_cast<const uint16_t *>(vals);
+    const long half_c = C / 2, meta_c = C / 8;
+    // values: 128 rows x 8 chunks
+    for (int i = threadIdx.x; i < 128 * 8; i += 256) {
+        const int r = i >> 3, q = i & 7;
+        const long row = (long)ft * 128 + r;
+        const long col = (long)kt * 64 + q * 8;      // in kept-value units
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row < No && col + 8 <= half_c) {
+            v = *reinterpret_cast<const uint4 *>(v16 + row * half_c + col);
+        } else if (row < No && col < half_c) {
+            uint16_t *p = reinterpret_cast<uint16_t *>(&v);
+            for (int e = 0; e < 8; ++e) if (col + e < half_c) p[e] = v16[row * half_c + col + e];
+        }
+        *reinterpret_cast<uint4 *>(tile + r * 128 + ((q ^ (r & 7)) << 4)) = v;
+    }
+    // metadata: 128 lanes x 4 words
+    for (int i = threadIdx.x; i < 128 * 4; i += 256) {
+        const int l = i >> 2, c = i & 3;
+        const int r_lo = (l & 7) + 16 * (l >> 4);
+        const int khalf = (l >> 3) & 1;
+        unsigned int word = 0;
+#pragma unroll
+        for (int hi = 0; hi < 2; ++hi) {
+            const long row = (long)ft * 128 + r_lo + 8 * hi;
+            const long mb = (long)kt * 16 + c * 4 + khalf * 2;   // metadata byte column
+            unsigned int m16 = 0x4444u;                          // padding: legal nibbles, values are zero
+            if (row < No) {
+                unsigned int b0 = (mb < meta_c) ? meta[row * meta_c + mb] : 0x44u;
+                unsigned int b1 = (mb + 1 < meta_c) ? meta[row * meta_c + mb + 1] : 0x44u;
+                m16 = b0 | (b1 << 8);
+            }
+            word |= m16 << (16 * hi);
+        }
+        reinterpret_cast<unsigned int *>(tile + kTileValBytes)[l * 4 + c] = word;
+    }
+}
+
+// K11: dense [No, C] in original channel order, zeros where pruned.
+__global__ void __launch_bounds__(256) decompress_kernel(const __half *__restrict__ vals, const uint8_t *__restrict__ meta,
+                                                         const int32_t *__restrict__ perm, int No, int C,
+                                                         __half *__restrict__ out, long ldw) {
+    const int j = blockIdx.x;
+    const uint16_t *v16 = reinterpret_cast<const uint16_t *>(vals) + (long)j * (C / 2);
+    uint16_t *o = reinterpret_cast<uint16_t *>(out) + (long)j * ldw;
+    for (int g = threadIdx.x; g < C / 4; g += 256) {
+        unsigned int byte = meta[(long)j * (C / 8) + (g >> 1)];
+        unsigned int nib = (g & 1) ? (byte >> 4) : (byte & 0xF);
+        int i0 = nib & 3, i1 = (nib >> 2) & 3;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int c = perm ? perm[4 * g + k] : 4 * g + k;
+            uint16_t v = 0;
+            if (k == i0) v = v16[2 * g];
+            if (k == i1) v = v16[2 * g + 1];
+            o[c] = v;
+        }
+    }
+}
+
+}  // namespace
+
+// ----------------------------------------------------------------------------------------------------
+// Host side
+// ----------------------------------------------------------------------------------------------------
+static int pick_splits(int rows, int col_blocks, int sm_count) {
+    // enough CTAs to fill the machine a few times over, each with a worthwhile slice of rows
+    int want = ceil_div(4L * sm_count, col_blocks);
+    int max_by_rows = ceil_div(rows, 64);
+    int s = want < 1 ? 1 : want;
+    if (s > max_by_rows) s = max_by_rows;
+    if (s > 1024) s = 1024;
+    return s < 1 ? 1 : s;
+}
+
+PruneWorkspace carve_prune_workspace(void *ws, int No, int C, int T, const esp_prune_opts &o) {
+    PruneWorkspace w{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { void *p = ws ? (char *)ws + off : nullptr; off += align_up(bytes, 256); return p; };
+    // the split count must not depend on the device so the size query and the call agree
+    w.splits = ceil_div(T > 0 ? T : 1, 256);
+    if (w.splits > 64) w.splits = 64;
+    w.part_sumsq = (double *)take(sizeof(double) * (size_t)w.splits * C);
+    w.part_min = (float *)take(sizeof(float) * (size_t)w.splits * C);
+    w.part_max = (float *)take(sizeof(float) * (size_t)w.splits * C);
+    w.lo = (double *)take(sizeof(double) * C);
+    w.hi = (double *)take(sizeof(double) * C);
+    w.norm = (double *)take(sizeof(double) * C);
+    w.entropy = (double *)take(sizeof(double) * C);
+    w.score = (double *)take(sizeof(double) * C);
+    w.mean = (double *)take(sizeof(double) * C);
+    w.counts = (unsigned int *)take(sizeof(unsigned int) * (size_t)C * o.bins);
+    w.colsum = (unsigned long long *)take(sizeof(unsigned long long) * C);
+    w.theta0 = (int32_t *)take(sizeof(int32_t) * C);
+    w.counters = (unsigned long long *)take(sizeof(unsigned long long) * 8);
+    w.objective = (double *)take(sizeof(double) * 2);
+    w.ldt = (long)align_up((size_t)No, 256);
+    w.wt = (uint16_t *)take(sizeof(uint16_t) * (size_t)C * w.ldt);
+    int nblocks = ceil_div(C, o.lbs_block > 0 ? o.lbs_block : kLbsMax);
+    w.table = (double *)take(sizeof(double) * (size_t)nblocks * kLbsGroups * 4 * kLbsMax);
+    w.base = (double *)take(sizeof(double) * (size_t)(C / 4 + 1));
+    w.total_bytes = off;
+    return w;
+}
+
+esp_status_t launch_pack(const __half *vals, const uint8_t *meta, int No, int C, void *packed, cudaStream_t stream) {
+    const int k_tiles = ceil_div(C, kTileK), f_tiles = ceil_div(No, kTileFeat);
+    pack_kernel<<<dim3(k_tiles, f_tiles), 256, 0, stream>>>(vals, meta, No, C, (uint8_t *)packed, k_tiles);
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+esp_status_t launch_decompress(const __half *vals, const uint8_t *meta, const int32_t *perm, int No, int C,
+                               __half *out, long ldw, cudaStream_t stream) {
+    decompress_kernel<<<No, 256, 0, stream>>>(vals, meta, perm, No, C, out, ldw);
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half *Xcal, int T, long ldx,
+                          const esp_prune_opts &o, __half *vals, uint8_t *meta, int32_t *perm, void *packed,
+                          double *chan_norm, double *chan_entropy, double *chan_score, esp_prune_stats *stats,
+                          PruneWorkspace &w, cudaStream_t stream) {
+    DeviceInfo di;
+    esp_status_t st = device_info(&di);
+    if (st != ESP_OK) return st;
+    const int cthreads = 256;
+    const int cblocks = ceil_div(C, cthreads);
+    ESP_CUDA_OK(cudaMemsetAsync(w.counters, 0, sizeof(unsigned long long) * 8, stream));
+    ESP_CUDA_OK(cudaMemsetAsync(w.objective, 0, sizeof(double) * 2, stream));
+
+    const bool need_stats_pass = (o.score_override == nullptr) || chan_norm || chan_entropy;
+    if (need_stats_pass && Xcal) {
+        // K1
+        const int rows1 = ceil_div(T, w.splits);
+        colstats_kernel<<<dim3(ceil_div(C, 256), w.splits), 256, 0, stream>>>(Xcal, T, C, ldx, rows1, w.part_sumsq,
+                                                                             w.part_min, w.part_max);
+        colstats_finish_kernel<<<cblocks, cthreads, 0, stream>>>(C, w.splits, w.part_sumsq, w.part_min, w.part_max,
+                                                                 w.norm, w.lo, w.hi);
+        // K2
+        ESP_CUDA_OK(cudaMemsetAsync(w.counts, 0, sizeof(unsigned int) * (size_t)C * o.bins, stream));
+        const int hsplits = pick_splits(T, ceil_div(C, 64), di.sm_count);
+        const int rows2 = ceil_div(T, hsplits);
+        const size_t hsmem = sizeof(unsigned int) * 64 * (size_t)o.bins;
+        ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem));
+        histogram_kernel<<<dim3(ceil_div(C, 64), hsplits), 256, hsmem, stream>>>(Xcal, T, C, ldx, rows2, o.bins, w.lo,
+                                                                                 w.hi, w.counts);
+        entropy_score_kernel<<<cblocks, cthreads, 0, stream>>>(C, T, o.bins, w.counts, w.norm, o.alpha, o.use_entropy,
+                                                               o.use_norm, o.score_override, w.entropy, w.score);
+    } else {
+        entropy_score_kernel<<<cblocks, cthreads, 0, stream>>>(C, T, o.bins, nullptr, w.norm, o.alpha, o.use_entropy,
+                                                               o.use_norm, o.score_override, w.entropy, w.score);
+    }
+    ESP_CUDA_OK(cudaGetLastError());
+    if (chan_norm) ESP_CUDA_OK(cudaMemcpyAsync(chan_norm, w.norm, sizeof(double) * C, cudaMemcpyDeviceToDevice, stream));
+    if (chan_entropy) ESP_CUDA_OK(cudaMemcpyAsync(chan_entropy, w.entropy, sizeof(double) * C, cudaMemcpyDeviceToDevice, stream));
+    if (chan_score) ESP_CUDA_OK(cudaMemcpyAsync(chan_score, w.score, sizeof(double) * C, cudaMemcpyDeviceToDevice, stream));
+
+    // K3 + K4
+    if (o.use_gns) {
+        ESP_CUDA_OK(cudaMemsetAsync(w.colsum, 0, sizeof(unsigned long long) * C, stream));
+        const int wsplits = pick_splits(No, ceil_div(C, 256), di.sm_count);
+        colabs_kernel<<<dim3(ceil_div(C, 256), wsplits), 256, 0, stream>>>(W, No, C, ldw, ceil_div(No, wsplits), w.colsum);
+        mean_metric_kernel<<<cblocks, cthreads, 0, stream>>>(C, No, w.colsum, w.score, w.mean);
+    }
+    int32_t *theta0 = (o.use_lbs || stats) ? w.theta0 : perm;
+    gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, theta0);
+    ESP_CUDA_OK(cudaGetLastError());
+
+    // K5
+    const int G = C / 4;
+    if (o.use_lbs || stats) {
+        abs_transpose_kernel<<<dim3(ceil_div(C, 32), ceil_div(w.ldt, 32)), 256, 0, stream>>>(W, No, C, ldw, w.wt, w.ldt);
+    }
+    if (o.use_lbs) {
+        const int nblocks = ceil_div(C, o.lbs_block);
+        lbs_table_kernel<<<nblocks * kLbsGroups, 256, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, C, o.lbs_block,
+                                                                  w.table, w.base);
+        if (stats) objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective);
+        lbs_greedy_kernel<<<nblocks, 512, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, C, o.lbs_block, o.lbs_max_swaps,
+                                                        w.table, w.base, perm, w.counters);
+        if (stats) objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective + 1);
+    } else if (stats) {
+        group_values_kernel<<<ceil_div(G, 8), 256, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, G, w.base);
+        objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective);
+        ESP_CUDA_OK(cudaMemcpyAsync(w.objective + 1, w.objective, sizeof(double), cudaMemcpyDeviceToDevice, stream));
+        ESP_CUDA_OK(cudaMemcpyAsync(perm, w.theta0, sizeof(int32_t) * C, cudaMemcpyDeviceToDevice, stream));
+    }
+    ESP_CUDA_OK(cudaGetLastError());
+
+    // K6 + K7
+    const size_t row_smem = sizeof(uint16_t) * (size_t)C;
+    ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_smem));
+    select_compress_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
+    ESP_CUDA_OK(cudaGetLastError());
+    if (packed) {
+        st = launch_pack(vals, meta, No, C, packed, stream);
+        if (st != ESP_OK) return st;
+    }
+    if (stats) {
+        unsigned long long h_counters[8];
+        double h_obj[2];
+        ESP_CUDA_OK(cudaMemcpyAsync(h_counters, w.counters, sizeof(h_counters), cudaMemcpyDeviceToHost, stream));
+        ESP_CUDA_OK(cudaMemcpyAsync(h_obj, w.objective, sizeof(h_obj), cudaMemcpyDeviceToHost, stream));
+        ESP_CUDA_OK(cudaStreamSynchronize(stream));
+        stats->near_tie_groups = (long long)h_counters[0];
+        stats->lbs_swaps_total = (long long)h_counters[1];
+        stats->obj_after_gns = h_obj[0];
+        stats->obj_after_lbs = h_obj[1];
+    }
+    return ESP_OK;
+}
+
+}  // namespace esp

@@ -1,0 +1,427 @@
+// esp_spgemm: Y = X . P . W_s^T on the 5th-generation tensor cores with the sparse-operand MMA
+// ("Efficient Sparse-GEMM Implementation": the product every pruned linear layer runs).
+//
+// Orientation.  The sparse operand must be the MMA's A operand, so each CTA computes a tile of Y^T:
+//   D[feature (128 TMEM lanes), token (TMEM columns)] += Wc[feature, k/2] (sparse, metadata in TMEM) * Xp[k, token]
+// The compressed weight arrives as pre-swizzled 18 KB tiles (16 KB values + 2 KB metadata), one bulk
+// async copy per pipeline stage; the metadata is copied shared -> tensor memory with tcgen05.cp right
+// before the four K=32 MMAs of a 128-channel tile.  The permutation P is applied while the X tile is
+// brought into shared memory (element gather in this file), never as a separate pass over X.
+// K is split across the CTAs of a thread-block cluster; partial tiles are summed in slice order through
+// distributed shared memory, so no global scratch is used and the result is deterministic.
+#include "esp_common.cuh"
+
+namespace esp {
+namespace {
+
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct GemmParams {
+    const __half *X;
+    long ldx;
+    int M, K, N;
+    int x_channel_major;
+    const uint8_t *packed;
+    const int32_t *perm;
+    void *Y;
+    long ldy;
+    int out_f32;
+    int k_tiles;             // ceil(K / 128)
+    int k_tiles_per_split;
+};
+
+// ---------------------------------------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or when another thread of the CTA gave up), records
+// ESP_ERR_TIMEOUT in the device status word and lets the caller fall through to the common exit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 128) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// shared memory (128 rows x 16 bytes, rows 16 bytes apart) -> 4 tensor-memory columns of all 128 lanes
+__device__ __forceinline__ void tc_copy_128x128b(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// D[tmem] (+)= A_sparse[smem] * B[smem], fp16 inputs, K = 32 channels (16 stored values per row of A)
+__device__ __forceinline__ void tc_mma_sparse_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t e_tmem,
+                                                  uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_load_16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// Shared-memory matrix descriptor of the tensor-core instructions (address, leading / stride byte
+// offsets in 16-byte units, descriptor version 1, swizzle mode in the top bits).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)layout << 61;
+    return d;
+}
+constexpr uint32_t kLayoutNone = 0, kLayoutSw128 = 2;
+
+// Instruction descriptor, kind::f16: sparse flag (bit 2), fp32 accumulator (bits 4-5 = 1), fp16 A and B
+// (formats 0), A K-major, B major as given (bit 16), N >> 3 (bits 17-22), M >> 4 (bits 24-28).
+__host__ __device__ constexpr uint32_t instr_desc_sparse_f16(int mma_m, int mma_n, int b_mn_major) {
+    return (1u << 2) | (1u << 4) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(mma_n >> 3) << 17) |
+           ((uint32_t)(mma_m >> 4) << 24);
+}
+
+__host__ __device__ constexpr int tmem_cols_for(int bn) { return bn + 8 <= 32 ? 32 : bn + 8 <= 64 ? 64 : bn + 8 <= 128 ? 128 : bn + 8 <= 256 ? 256 : 512; }
+
+template <int BN, int STAGES>
+struct GatherSmem {
+    static constexpr int kWBytes = STAGES * kTileBytes;
+    static constexpr int kXStage = BN * 256;                   // BN tokens x 128 channels fp16
+    static constexpr int kXBytes = STAGES * kXStage;
+    static constexpr int kStageArea = kWBytes + kXBytes;
+    static constexpr int kReduceBytes = BN * 128 * 4;          // fp32 partial tile, aliases the stage area
+    static constexpr int kMain = kStageArea > kReduceBytes ? kStageArea : kReduceBytes;
+    static constexpr int kBarOff = kMain;                      // barriers, TMEM slot, abort flag
+    static constexpr int kTotal = kBarOff + 256 + 1024;        // + slack for 1024-byte alignment of the base
+};
+
+// --------------------------------------------------------------------------------------------------
+// Gather kernel: any M, either X layout; the X tile is gathered element-wise through the permutation by
+// four warps.  Used for decode shapes (X is tiny and cache resident, the weight stream is the cost).
+// grid (feature tiles, token tiles, split_k), cluster (1, 1, split_k), block 192:
+//   warp 0 lane 0  weight-tile producer (bulk async copies)      warp 1 lane 0  MMA issuer
+//   warps 2..5     X gather producers, then epilogue (one TMEM lane quarter each)
+// --------------------------------------------------------------------------------------------------
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(192) spgemm_gather_kernel(const GemmParams p) {
+    using L = GatherSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t w_base = sbase, x_base = sbase + L::kWBytes;
+    const uint32_t bar_base = sbase + L::kBarOff;
+    auto full_w = [&](int s) { return bar_base + 8u * s; };
+    auto full_x = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto empty = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
+    const uint32_t accum_bar = bar_base + 8u * (3 * STAGES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * (3 * STAGES + 1));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * (3 * STAGES + 1) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
+    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
+    const int kt_begin = slice * p.k_tiles_per_split;
+    const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
+    const int nk = max(0, kt_end - kt_begin);
+    constexpr uint32_t kTmemCols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_w(s), 1);
+            mbar_init(full_x(s), 4);
+            mbar_init(empty(s), 1);
+        }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint8_t *src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(full_w(s), kTileBytes);
+                bulk_load(w_base + s * kTileBytes, src + (long)it * kTileBytes, kTileBytes, full_w(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 0);
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(full_w(s), ph, abort_flag)) break;
+                if (!mbar_wait(full_x(s), ph, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t wa = w_base + s * kTileBytes;
+                const uint32_t xa = x_base + s * L::kXStage;
+                const uint32_t e_col = BN + (it & 1) * 4;
+                tc_copy_128x128b(tmem + e_col, smem_desc(wa + kTileValBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t col = e_col + j;
+                    const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
+                    const uint64_t bd = smem_desc(xa + (j >> 1) * (BN * 128) + (j & 1) * 64, 16, 1024, kLayoutSw128);
+                    tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            tc_commit(accum_bar);
+        }
+    } else {
+        // ---- X gather: thread g owns channel chunk (g & 15) of tokens (g >> 4) + 8 i
+        const int g = threadIdx.x - 64;
+        const int chunk = g & 15;
+        bool alive = true;
+        for (int it = 0; it < nk && alive; ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+            const int kc = (kt_begin + it) * kTileK + chunk * 8;
+            int th[8];
+            if (kc + 8 <= p.K && p.perm) {
+                const int4 a = __ldg(reinterpret_cast<const int4 *>(p.perm + kc));
+                const int4 b = __ldg(reinterpret_cast<const int4 *>(p.perm + kc + 4));
+                th[0] = a.x; th[1] = a.y; th[2] = a.z; th[3] = a.w;
+                th[4] = b.x; th[5] = b.y; th[6] = b.z; th[7] = b.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) th[e] = (kc + e < p.K) ? (p.perm ? p.perm[kc + e] : kc + e) : -1;
+            }
+            uint8_t *xs = smem + L::kWBytes + s * L::kXStage + (chunk >> 3) * (BN * 128);
+            const int q = chunk & 7;
+            for (int row = g >> 4; row < BN; row += 8) {
+                const int t = tok0 + row;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (t < p.M) {
+                    uint16_t h[8];
+                    const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        long off = p.x_channel_major ? ((long)th[e] * p.ldx + t) : ((long)t * p.ldx + th[e]);
+                        h[e] = th[e] >= 0 ? __ldg(xb + off) : (uint16_t)0;
+                    }
+                    v.x = h[0] | ((uint32_t)h[1] << 16);
+                    v.y = h[2] | ((uint32_t)h[3] << 16);
+                    v.z = h[4] | ((uint32_t)h[5] << 16);
+                    v.w = h[6] | ((uint32_t)h[7] << 16);
+                }
+                *reinterpret_cast<uint4 *>(xs + row * 128 + ((q ^ (row & 7)) << 4)) = v;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full_x(s));
+        }
+        // ---- epilogue: TMEM lane quarter (warp & 3)
+        const int quarter = warp & 3;
+        const int f_local = quarter * 32 + lane;
+        const long feature = (long)ft * 128 + f_local;
+        bool ok = alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
+        tc_fence_after();
+        float *stage_f32 = reinterpret_cast<float *>(smem);
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            uint32_t v[16];
+            if (nk > 0) {
+                tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0;
+            }
+            if (split == 1) {
+                if (ok && feature < p.N) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int t = tok0 + c0 + e;
+                        if (t < p.M) {
+                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
+                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
+                        }
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+            }
+        }
+        tc_fence_before();
+    }
+
+    if (split > 1) {
+        // all partial tiles are in shared memory: sum them in slice order, each CTA finishing 1/split of the tokens
+        cluster_sync_all();
+        const uint32_t rank = cluster_ctarank();
+        const bool ok = (*abort_flag == 0);
+        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
+            const int row = idx >> 7, f_local = idx & 127;
+            if ((row % split) != (int)rank) continue;
+            const int t = tok0 + row;
+            const long feature = (long)ft * 128 + f_local;
+            if (t >= p.M || feature >= p.N) continue;
+            float acc = 0.f;
+            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
+            if (ok) {
+                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
+                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
+            }
+        }
+        cluster_sync_all();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+template <int BN, int STAGES>
+esp_status_t launch_gather(const GemmParams &p, int f_tiles, int t_tiles, int split, cudaStream_t stream) {
+    using L = GatherSmem<BN, STAGES>;
+    auto kern = spgemm_gather_kernel<BN, STAGES>;
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(f_tiles, t_tiles, split);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
+    return ESP_OK;
+}
+
+}  // namespace
+
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, GemmPlan *plan) {
+    DeviceInfo di;
+    esp_status_t st = device_info(&di);
+    if (st != ESP_OK) return st;
+    GemmPlan g;
+    g.kernel = ESP_KERNEL_GATHER;
+    int bn = o.token_tile;
+    if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
+    g.token_tile = bn;
+    const int k_tiles = ceil_div(K, kTileK);
+    const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, bn);
+    int split = o.split_k;
+    if (split == 0) {
+        split = 1;
+        while (split < 8 && (long)f_tiles * t_tiles * split < di.sm_count && k_tiles / (split * 2) >= 4) split *= 2;
+    }
+    if (split > k_tiles) split = k_tiles;
+    if (split < 1) split = 1;
+    // every slice must own at least one tile
+    while (split > 1 && (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles) --split;
+    g.split_k = split;
+    g.stages = 4;
+    *plan = g;
+    return ESP_OK;
+}
+
+esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
+                           void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan, void *workspace,
+                           size_t workspace_bytes, cudaStream_t stream) {
+    (void)workspace; (void)workspace_bytes;
+    GemmParams p;
+    p.X = X; p.ldx = ldx; p.M = M; p.K = K; p.N = N;
+    p.x_channel_major = (o.x_layout == ESP_X_CHANNEL_MAJOR) ? 1 : 0;
+    p.packed = (const uint8_t *)packed;
+    p.perm = perm;
+    p.Y = Y; p.ldy = ldy;
+    p.out_f32 = (o.out_dtype == ESP_OUT_F32) ? 1 : 0;
+    p.k_tiles = ceil_div(K, kTileK);
+    p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
+    const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
+    switch (plan.token_tile) {
+        case 16: return launch_gather<16, 6>(p, f_tiles, t_tiles, plan.split_k, stream);
+        case 32: return launch_gather<32, 6>(p, f_tiles, t_tiles, plan.split_k, stream);
+        case 64: return launch_gather<64, 5>(p, f_tiles, t_tiles, plan.split_k, stream);
+        case 128: return launch_gather<128, 4>(p, f_tiles, t_tiles, plan.split_k, stream);
+        case 256: return launch_gather<256, 2>(p, f_tiles, t_tiles, plan.split_k, stream);
+        default: return ESP_ERR_INVALID_ARG;
+    }
+}
+
+}  // namespace esp
