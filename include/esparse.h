@@ -135,7 +135,11 @@ enum { ESP_X_TOKEN_MAJOR = 0,    /* X[t, c] at X + t * ldx + c  (tokens are rows
        ESP_X_CHANNEL_MAJOR = 1 };/* X[t, c] at X + c * ldx + t  (channels are rows: the activation
                                     handed over transposed)                                           */
 enum { ESP_OUT_F16 = 0, ESP_OUT_F32 = 1 };
-enum { ESP_KERNEL_AUTO = 0, ESP_KERNEL_GATHER = 1, ESP_KERNEL_TMA = 2 };
+enum { ESP_KERNEL_AUTO = 0,
+       ESP_KERNEL_GATHER = 1,    /* element gather of X, any layout, no workspace (slow for large M)    */
+       ESP_KERNEL_TMA = 2,       /* channel-major X tiles fetched row-wise by the tensor memory unit    */
+       ESP_KERNEL_RESIDENT = 3 };/* small M: the CTA's whole K-slice of X is gathered once, then only
+                                    weight tiles stream                                                 */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
@@ -148,7 +152,11 @@ typedef struct {
 
 void esp_gemm_opts_default(esp_gemm_opts *opts);
 
-/* Bytes of device workspace esp_spgemm needs (may be 0; then workspace may be NULL). */
+/*
+ * Bytes of device workspace esp_spgemm can use.  0 for channel-major X.  For token-major X it is the size
+ * of a transposed (channels-as-rows, not permuted) copy of X, which lets the fast kernels run; with a NULL
+ * or smaller workspace the call still works through the element-gather kernel.
+ */
 size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts);
 
 /*

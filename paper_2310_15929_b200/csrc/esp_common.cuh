@@ -66,12 +66,13 @@ esp_status_t launch_decompress(const __half *vals, const uint8_t *meta, const in
 
 // ---- GEMM launchers (spgemm_kernels.cu) ------------------------------------------------------------
 struct GemmPlan {
-    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA
+    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_RESIDENT | ESP_KERNEL_TMA
     int token_tile;    // MMA N
     int split_k;       // cluster size along K
     int stages;
 };
-esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, GemmPlan *plan);
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan);
+size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o);
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm,
                            int N, void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan,
                            void *workspace, size_t workspace_bytes, cudaStream_t stream);

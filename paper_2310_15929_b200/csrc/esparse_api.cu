@@ -41,7 +41,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->x_layout != ESP_X_TOKEN_MAJOR && o->x_layout != ESP_X_CHANNEL_MAJOR) return ESP_ERR_INVALID_ARG;
     if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
-    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_TMA) return ESP_ERR_INVALID_ARG;
+    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_RESIDENT) return ESP_ERR_INVALID_ARG;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
 }
@@ -146,8 +146,11 @@ esp_status_t esp_decompress(const void *vals, const void *meta, const int32_t *p
 }
 
 size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts) {
-    (void)M; (void)N; (void)K; (void)opts;
-    return 0;   // K-slices are reduced through distributed shared memory inside a cluster: no global scratch
+    (void)N;
+    if (M <= 0 || K <= 0 || check_gemm_opts(opts) != ESP_OK) return 0;
+    // K-slices are reduced through distributed shared memory inside a cluster: no global scratch for that.
+    // Token-major X is first transposed (not permuted) into the workspace so channels become rows.
+    return gemm_workspace_bytes(M, K, *opts);
 }
 
 esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
@@ -165,7 +168,8 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packe
     if (st != ESP_OK) return st;
     if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
     GemmPlan plan;
-    st = plan_gemm(M, N, K, *opts, &plan);
+    const bool have_ws = workspace && workspace_bytes >= gemm_workspace_bytes(M, K, *opts) && aligned16(workspace);
+    st = plan_gemm(M, N, K, *opts, have_ws, &plan);
     if (st != ESP_OK) return st;
     return launch_spgemm((const __half *)X, M, K, ldx, packed, perm, N, Y, ldy, *opts, plan, workspace,
                          workspace_bytes, (cudaStream_t)cuda_stream);

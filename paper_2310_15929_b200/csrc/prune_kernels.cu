@@ -530,7 +530,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const __half *__restrict__ va
         const long row = (long)ft * 128 + r;
         const long col = (long)kt * 64 + q * 8;      // in kept-value units
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (row < No && col + 8 <= half_c) {
+        if (row < No && col + 8 <= half_c && (half_c & 7) == 0) {      // rows of vals are 16-byte aligned
             v = *reinterpret_cast<const uint4 *>(v16 + row * half_c + col);
         } else if (row < No && col < half_c) {
             uint16_t *p = reinterpret_cast<uint16_t *>(&v);

@@ -371,31 +371,293 @@ esp_status_t launch_gather(const GemmParams &p, int f_tiles, int t_tiles, int sp
     return ESP_OK;
 }
 
+
+// --------------------------------------------------------------------------------------------------
+// Resident-X kernel: small token counts (decode), channel-major X.
+// Each CTA owns a feature tile and a K-slice.  Its whole slice of permuted X (BN tokens per channel, one
+// swizzled shared-memory row per channel: an MN-major B operand) is gathered once at start-up by all
+// threads with 16-byte loads -- one or two sectors per channel, all loads independent -- while the first
+// weight tiles are already in flight; afterwards the main loop only streams compressed weight tiles
+// (one 18 KB bulk copy per stage), which is the HBM-bound part.
+// grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192.
+// --------------------------------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(192) spgemm_resident_kernel(const GemmParams p, const int stages) {
+    constexpr int RB = BN * 2;                       // bytes of one channel row of the X tile
+    constexpr int kXTile = 128 * RB;                 // one 128-channel tile of X
+    constexpr uint32_t kLayout = (BN == 16) ? 6u : (BN == 32) ? 4u : 2u;   // 32 / 64 / 128-byte swizzle
+    constexpr int kSwzShift = (BN == 16) ? 2 : (BN == 32) ? 1 : 0;         // row bits that feed the XOR
+    constexpr int kChunks = RB / 16;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
+    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
+    const int kt_begin = slice * p.k_tiles_per_split;
+    const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
+    const int nk = max(0, kt_end - kt_begin);
+
+    const uint32_t w_base = sbase;                                   // stages x 18432
+    const uint32_t x_base = sbase + (uint32_t)stages * kTileBytes;   // k_tiles_per_split x kXTile
+    const uint32_t bar_base = x_base + (uint32_t)p.k_tiles_per_split * kXTile;
+    uint8_t *bar_ptr = smem + (size_t)stages * kTileBytes + (size_t)p.k_tiles_per_split * kXTile;
+    auto full_w = [&](int s) { return bar_base + 8u * s; };
+    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
+    const uint32_t accum_bar = bar_base + 8u * 16;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_ptr + 8 * 17);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_ptr + 8 * 17 + 4);
+    constexpr uint32_t kTmemCols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(full_w(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
+
+    // first weight tiles go out before the X gather so the two latencies overlap
+    const int prefetch = min(stages, nk);
+    if (threadIdx.x == 0) {
+        for (int it = 0; it < prefetch; ++it) {
+            mbar_arrive_expect_tx(full_w(it), kTileBytes);
+            bulk_load(w_base + it * kTileBytes, w_src + (long)it * kTileBytes, kTileBytes, full_w(it));
+        }
+    }
+    // gather the K-slice of X: one channel row per iteration per thread
+    {
+        const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
+        for (int r = threadIdx.x; r < nk * 128; r += 192) {
+            const int kpos = kt_begin * kTileK + r;
+            int ch = -1;
+            if (kpos < p.K) ch = p.perm ? __ldg(p.perm + kpos) : kpos;
+            uint8_t *row = smem + (size_t)stages * kTileBytes + (size_t)r * RB;
+            const int rr = r & 127;
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c) {
+                uint4 v = make_uint4(0, 0, 0, 0);
+                const int t = tok0 + c * 8;
+                if (ch >= 0) {
+                    const uint16_t *src = xb + (long)ch * p.ldx + t;
+                    if (t + 8 <= p.M) {
+                        v = __ldg(reinterpret_cast<const uint4 *>(src));
+                    } else if (t < p.M) {
+                        uint16_t h[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) h[e] = (t + e < p.M) ? __ldg(src + e) : (uint16_t)0;
+                        v.x = h[0] | ((uint32_t)h[1] << 16); v.y = h[2] | ((uint32_t)h[3] << 16);
+                        v.z = h[4] | ((uint32_t)h[5] << 16); v.w = h[6] | ((uint32_t)h[7] << 16);
+                    }
+                }
+                const int cs = c ^ ((rr >> kSwzShift) & (kChunks - 1));
+                *reinterpret_cast<uint4 *>(row + cs * 16) = v;
+            }
+        }
+        fence_async_smem();
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = prefetch; it < nk; ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(full_w(s), kTileBytes);
+                bulk_load(w_base + s * kTileBytes, w_src + (long)it * kTileBytes, kTileBytes, full_w(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                if (!mbar_wait(full_w(s), ph, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t wa = w_base + s * kTileBytes;
+                const uint32_t xa = x_base + it * kXTile;
+                const uint32_t e_col = BN + (it & 1) * 4;
+                tc_copy_128x128b(tmem + e_col, smem_desc(wa + kTileValBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t col = e_col + j;
+                    const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
+                    const uint64_t bd = smem_desc(xa + j * 32 * RB, 8 * RB, 8 * RB, kLayout);
+                    tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            tc_commit(accum_bar);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int f_local = quarter * 32 + lane;
+        const long feature = (long)ft * 128 + f_local;
+        const bool ok = (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
+        tc_fence_after();
+        float *stage_f32 = reinterpret_cast<float *>(smem);
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            uint32_t v[16];
+            if (nk > 0) {
+                tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0;
+            }
+            if (split == 1) {
+                if (ok && feature < p.N) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int t = tok0 + c0 + e;
+                        if (t < p.M) {
+                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
+                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
+                        }
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+            }
+        }
+        tc_fence_before();
+    }
+
+    if (split > 1) {
+        cluster_sync_all();
+        const uint32_t rank = cluster_ctarank();
+        const bool ok = (*abort_flag == 0);
+        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
+            const int row = idx >> 7, f_local = idx & 127;
+            if ((row % split) != (int)rank) continue;
+            const int t = tok0 + row;
+            const long feature = (long)ft * 128 + f_local;
+            if (t >= p.M || feature >= p.N) continue;
+            float acc = 0.f;
+            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
+            if (ok) {
+                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
+                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
+            }
+        }
+        cluster_sync_all();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+inline size_t resident_smem_bytes(int bn, int stages, int k_tiles_per_split) {
+    return (size_t)stages * kTileBytes + (size_t)k_tiles_per_split * 128 * bn * 2 + 256 + 1024;
+}
+
+template <int BN>
+esp_status_t launch_resident(const GemmParams &p, int f_tiles, int t_tiles, int split, int stages, cudaStream_t stream) {
+    auto kern = spgemm_resident_kernel<BN>;
+    const size_t smem = resident_smem_bytes(BN, stages, p.k_tiles_per_split);
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(f_tiles, t_tiles, split);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, stages));
+    return ESP_OK;
+}
+
+// [M, K] token-major -> [K, ldt] channel-major (a transposed, not permuted, copy; ldt >= M).
+__global__ void __launch_bounds__(256) transpose_x_kernel(const uint16_t *__restrict__ X, int M, int K, long ldx,
+                                                          uint16_t *__restrict__ Xt, long ldt) {
+    __shared__ uint16_t tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int k0 = blockIdx.x * 32, m0 = blockIdx.y * 32;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 8 * i, k = k0 + tx;
+        tile[ty + 8 * i][tx] = (m < M && k < K) ? X[(long)m * ldx + k] : (uint16_t)0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int k = k0 + ty + 8 * i, m = m0 + tx;
+        if (k < K && m < ldt) Xt[(long)k * ldt + m] = tile[tx][ty + 8 * i];
+    }
+}
+
 }  // namespace
 
-esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, GemmPlan *plan) {
+static long transposed_ld(int M) { return (long)((M + 15) / 16 * 16); }
+
+size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
+    if (o.x_layout == ESP_X_CHANNEL_MAJOR || o.force_kernel == ESP_KERNEL_GATHER) return 0;
+    return align_up((size_t)K * (size_t)transposed_ld(M) * 2, 256);
+}
+
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan) {
     DeviceInfo di;
     esp_status_t st = device_info(&di);
     if (st != ESP_OK) return st;
     GemmPlan g;
-    g.kernel = ESP_KERNEL_GATHER;
+    const int k_tiles = ceil_div(K, kTileK);
+    const int f_tiles = ceil_div(N, kTileFeat);
+    const bool channel_major_available = (o.x_layout == ESP_X_CHANNEL_MAJOR) || have_workspace;
     int bn = o.token_tile;
+    g.kernel = ESP_KERNEL_GATHER;
+    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available && M <= 64 && (bn == 0 || bn <= 64))
+        g.kernel = ESP_KERNEL_RESIDENT;
     if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
-    const int k_tiles = ceil_div(K, kTileK);
-    const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, bn);
+    const int t_tiles = ceil_div(M, bn);
     int split = o.split_k;
-    if (split == 0) {
+    g.stages = 4;
+    if (g.kernel == ESP_KERNEL_RESIDENT) {
+        // the K-slice of X must fit beside the weight stages; more slices also spread the weight stream
+        const size_t x_cap = 64 * 1024;
+        int min_split = 1;
+        while (min_split < 8 && (size_t)ceil_div(k_tiles, min_split) * 128 * bn * 2 > x_cap) ++min_split;
+        if (split == 0) {
+            split = min_split;
+            while (split < 8 && (long)f_tiles * t_tiles * split < 2L * di.sm_count && ceil_div(k_tiles, split + 1) >= 2) ++split;
+        }
+        if (split < min_split) split = min_split;
+        if ((size_t)ceil_div(k_tiles, split) * 128 * bn * 2 > 96 * 1024) g.kernel = ESP_KERNEL_GATHER;
+    }
+    if (g.kernel == ESP_KERNEL_GATHER && split == 0) {
         split = 1;
         while (split < 8 && (long)f_tiles * t_tiles * split < di.sm_count && k_tiles / (split * 2) >= 4) split *= 2;
     }
     if (split > k_tiles) split = k_tiles;
     if (split < 1) split = 1;
-    // every slice must own at least one tile
-    while (split > 1 && (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles) --split;
+    while (split > 1 && (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles) --split;   // no empty slice
     g.split_k = split;
-    g.stages = 4;
+    if (g.kernel == ESP_KERNEL_RESIDENT) {
+        const size_t xbytes = (size_t)ceil_div(k_tiles, split) * 128 * bn * 2;
+        const long ctas = (long)f_tiles * t_tiles * split;
+        const size_t budget = (ctas > di.sm_count ? 112 : 220) * 1024 - 2048;
+        int stages = (int)((budget - (xbytes < budget ? xbytes : budget)) / kTileBytes);
+        if (stages > 8) stages = 8;
+        if (stages < 2) stages = 2;
+        g.stages = stages;
+    }
     *plan = g;
     return ESP_OK;
 }
@@ -403,7 +665,6 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, GemmPlan *pl
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
                            void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan, void *workspace,
                            size_t workspace_bytes, cudaStream_t stream) {
-    (void)workspace; (void)workspace_bytes;
     GemmParams p;
     p.X = X; p.ldx = ldx; p.M = M; p.K = K; p.N = N;
     p.x_channel_major = (o.x_layout == ESP_X_CHANNEL_MAJOR) ? 1 : 0;
@@ -414,6 +675,25 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.k_tiles = ceil_div(K, kTileK);
     p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
+    if (plan.kernel == ESP_KERNEL_RESIDENT) {
+        if (!p.x_channel_major) {
+            // token-major input: transposed (not permuted) copy into the caller's workspace
+            const long ldt = transposed_ld(M);
+            if (!workspace || workspace_bytes < (size_t)K * ldt * 2) return ESP_ERR_WORKSPACE;
+            transpose_x_kernel<<<dim3(ceil_div(K, 32), ceil_div(ldt, 32)), 256, 0, stream>>>(
+                reinterpret_cast<const uint16_t *>(X), M, K, ldx, reinterpret_cast<uint16_t *>(workspace), ldt);
+            ESP_CUDA_OK(cudaGetLastError());
+            p.X = reinterpret_cast<const __half *>(workspace);
+            p.ldx = ldt;
+            p.x_channel_major = 1;
+        }
+        switch (plan.token_tile) {
+            case 16: return launch_resident<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
+            case 32: return launch_resident<32>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
+            case 64: return launch_resident<64>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
+            default: return ESP_ERR_INVALID_ARG;
+        }
+    }
     switch (plan.token_tile) {
         case 16: return launch_gather<16, 6>(p, f_tiles, t_tiles, plan.split_k, stream);
         case 32: return launch_gather<32, 6>(p, f_tiles, t_tiles, plan.split_k, stream);

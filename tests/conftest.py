@@ -9,6 +9,11 @@ if ROOT not in sys.path:
 
 
 def pytest_configure(config):
+    # the shared library is a build product (kept out of git): compile it if missing or stale
+    from paper_2310_15929_b200.build import build
+    from oracle.esparse_oracle import build_c
+    build()
+    build_c()
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
 

@@ -1,0 +1,128 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the header
+declares, and rejects bad arguments before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2310_15929_b200 import binding as b
+from paper_2310_15929_b200.build import HEADER, LIB_PATH
+
+
+def header_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(esp_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(LIB_PATH)
+    names = header_functions()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(b.EXPORTS)
+
+
+def test_version_and_status_strings():
+    assert b.esp_version() >= 100
+    seen = {b.esp_status_string(i) for i in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert b.esp_status_string(99) == "unknown status"
+
+
+def test_defaults_follow_the_paper():
+    o = b.esp_prune_opts_default()
+    assert (o.bins, o.n_keep, o.m_group, o.lbs_block) == (100, 2, 4, 256)
+    assert o.use_entropy and o.use_norm and o.use_gns and o.use_lbs and o.lbs_max_swaps == 0
+    assert o.struct_size == ctypes.sizeof(b.esp_prune_opts)
+    g = b.esp_gemm_opts_default()
+    assert g.struct_size == ctypes.sizeof(b.esp_gemm_opts) and g.x_layout == b.ESP_X_TOKEN_MAJOR
+
+
+def test_size_queries():
+    assert b.esp_packed_bytes(128, 128) == 18432
+    assert b.esp_packed_bytes(4096, 4096) == 4096 * 4096 * 2 * 9 // 16        # 9/16 of dense
+    assert b.esp_packed_bytes(129, 136) == 4 * 18432                           # padded to 128-multiples
+    assert b.esp_packed_bytes(0, 128) == 0
+    o = b.esp_prune_opts_default()
+    small = b.esp_metric_prune_workspace_bytes(512, 512, 128, o)
+    big = b.esp_metric_prune_workspace_bytes(4096, 4096, 32768, o)
+    assert 0 < small < big
+    assert b.esp_metric_prune_workspace_bytes(512, 510, 128, o) == 0           # C % 8 != 0
+    assert b.esp_spgemm_workspace_bytes(16, 4096, 4096, b.esp_gemm_opts_default()) == 0
+
+
+A = 0x10000   # a fake, 16-byte aligned "device address": argument errors must be caught before any use
+
+
+def prune_call(**kw):
+    o = kw.pop("opts", b.esp_prune_opts_default())
+    a = dict(W=A, No=512, C=512, ldw=512, Xcal=A, T=128, ldx=512, opts=o, vals=A, meta=A, perm=A, packed=None,
+             chan_norm=None, chan_entropy=None, chan_score=None, stats=None, workspace=A, workspace_bytes=1 << 30,
+             stream=None)
+    a.update(kw)
+    return b.esp_metric_prune_raw(**a)
+
+
+def test_prune_argument_errors():
+    assert prune_call(W=None) == b.ESP_ERR_INVALID_ARG
+    assert prune_call(perm=None) == b.ESP_ERR_INVALID_ARG
+    assert prune_call(Xcal=None) == b.ESP_ERR_INVALID_ARG                      # no calibration and no override
+    assert prune_call(opts=None) == b.ESP_ERR_INVALID_ARG
+    assert prune_call(C=508, ldw=512) == b.ESP_ERR_SHAPE
+    assert prune_call(ldw=256) == b.ESP_ERR_SHAPE
+    assert prune_call(No=0) == b.ESP_ERR_SHAPE
+    assert prune_call(T=0) == b.ESP_ERR_SHAPE
+    assert prune_call(ldw=516) == b.ESP_ERR_ALIGNMENT
+    assert prune_call(W=A + 2) == b.ESP_ERR_ALIGNMENT
+    assert prune_call(workspace=None) == b.ESP_ERR_WORKSPACE
+    assert prune_call(workspace_bytes=16) == b.ESP_ERR_WORKSPACE
+    o = b.esp_prune_opts_default(); o.n_keep, o.m_group = 4, 8
+    assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED                         # 4:8 has no sparse MMA form
+    o = b.esp_prune_opts_default(); o.bins = 5000
+    assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED
+    o = b.esp_prune_opts_default(); o.lbs_block = 250
+    assert prune_call(opts=o) == b.ESP_ERR_INVALID_ARG
+    o = b.esp_prune_opts_default(); o.struct_size = 8
+    assert prune_call(opts=o) == b.ESP_ERR_INVALID_ARG
+    s = b.esp_prune_stats(); s.struct_size = 3
+    assert prune_call(stats=s) == b.ESP_ERR_INVALID_ARG
+
+
+def gemm_call(**kw):
+    o = kw.pop("opts", b.esp_gemm_opts_default())
+    a = dict(X=A, M=16, K=512, ldx=512, packed=A, perm=A, N=512, Y=A, ldy=512, opts=o, workspace=None,
+             workspace_bytes=0, stream=None)
+    a.update(kw)
+    return b.esp_spgemm_raw(**a)
+
+
+def test_gemm_argument_errors():
+    assert gemm_call(X=None) == b.ESP_ERR_INVALID_ARG
+    assert gemm_call(packed=None) == b.ESP_ERR_INVALID_ARG
+    assert gemm_call(opts=None) == b.ESP_ERR_INVALID_ARG
+    assert gemm_call(M=0) == b.ESP_ERR_SHAPE
+    assert gemm_call(K=508) == b.ESP_ERR_SHAPE
+    assert gemm_call(ldx=256) == b.ESP_ERR_SHAPE
+    assert gemm_call(ldy=100) == b.ESP_ERR_SHAPE
+    assert gemm_call(ldx=516) == b.ESP_ERR_ALIGNMENT
+    assert gemm_call(Y=A + 8) == b.ESP_ERR_ALIGNMENT
+    o = b.esp_gemm_opts_default(); o.x_layout = 7
+    assert gemm_call(opts=o) == b.ESP_ERR_INVALID_ARG
+    o = b.esp_gemm_opts_default(); o.split_k = 9
+    assert gemm_call(opts=o) == b.ESP_ERR_INVALID_ARG
+    o = b.esp_gemm_opts_default(); o.token_tile = 24
+    assert gemm_call(opts=o) == b.ESP_ERR_INVALID_ARG
+    o = b.esp_gemm_opts_default(); o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    assert gemm_call(opts=o, ldx=8) == b.ESP_ERR_SHAPE                          # channel-major needs ldx >= M
+
+
+def test_no_gpu_means_cuda_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    # valid arguments, no device: the call must fail loudly, never compute on the CPU
+    assert prune_call() in (b.ESP_ERR_CUDA, b.ESP_ERR_UNSUPPORTED)
+    assert gemm_call() in (b.ESP_ERR_CUDA, b.ESP_ERR_UNSUPPORTED)

@@ -1,0 +1,117 @@
+"""GPU parity of esp_spgemm against the CPU oracle's fp64 product, through the C ABI.
+
+Bars (the stated tolerances of the method's GEMM check): max-abs error <= 2e-2 and relative Frobenius
+error <= 1e-3 on the fp16 output wherever |y| < 64 (fp16 spacing above that exceeds the bound by itself),
+fp16 output within one fp16 ulp of the oracle everywhere, and the fp32-output variant within 2e-2 / 1e-5.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import esparse_oracle as orc
+from paper_2310_15929_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+REL_FRO = 1e-3
+
+
+def check(Y, Yref, f32=False):
+    Y = Y.astype(np.float64)
+    assert not np.isnan(Y).any()
+    rel = np.linalg.norm(Y - Yref) / max(np.linalg.norm(Yref), 1e-30)
+    assert rel <= (1e-5 if f32 else REL_FRO), rel
+    small = np.abs(Yref) < 64
+    assert np.abs(Y - Yref)[small].max(initial=0.0) <= MAX_ABS
+    if f32:
+        assert np.abs(Y - Yref).max() <= MAX_ABS
+    else:
+        ulp = np.spacing(np.abs(Yref).astype(np.float16)).astype(np.float64)
+        assert np.all(np.abs(Y - Yref) <= ulp + 1e-3 * np.abs(Yref) + 1e-4)
+
+
+def pruned(seed, N, K, T=64):
+    g = np.random.default_rng(seed)
+    W = (g.standard_normal((N, K)) * 0.02).astype(np.float16)
+    Xc = g.standard_normal((T, K)).astype(np.float16)
+    s = orc.channel_score(orc.channel_entropy(Xc), orc.channel_norm(Xc), 0.1)
+    theta = g.permutation(K).astype(np.int32)
+    vals, meta, _ = orc.select_compress(W, s, theta)
+    return vals, meta, theta
+
+
+def test_config0_all_variants():
+    from tests.gpu_util import pack_on_gpu, spgemm
+    wl = inputs.WORKLOADS[0]
+    W, Xc = inputs.make_weight(wl, "fc"), inputs.make_calibration(wl, "fc")
+    ref = orc.metric_prune(W, Xc, 1.0 / math.sqrt(128))
+    packed = pack_on_gpu(ref.vals, ref.meta)
+    X = inputs.make_gemm_x(wl, "fc", 128)
+    Yref = orc.product(X, ref.vals, ref.meta, ref.theta)
+    for kw in (dict(), dict(split_k=2), dict(split_k=4, out_f32=True), dict(channel_major=True),
+               dict(token_tile=64), dict(token_tile=16, split_k=4), dict(token_tile=256, out_f32=True),
+               dict(token_tile=64, channel_major=True, split_k=2), dict(token_tile=32, workspace=True),
+               dict(kernel=1, workspace=False), dict(kernel=1, channel_major=True, token_tile=128)):
+        check(spgemm(X, packed, ref.theta, 512, **kw), Yref, kw.get("out_f32", False))
+
+
+@pytest.mark.parametrize("M", [1, 4, 16, 17, 64, 130])
+@pytest.mark.parametrize("N,K", [(512, 512), (200, 264), (384, 1160)])
+def test_decode_and_ragged_shapes(M, N, K):
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(N * 7 + K, N, K)
+    X = np.random.default_rng(M).standard_normal((M, K)).astype(np.float16)
+    Yref = orc.product(X, vals, meta, theta)
+    packed = pack_on_gpu(vals, meta)
+    check(spgemm(X, packed, theta, N), Yref)                                   # token-major + transposed copy
+    check(spgemm(X, packed, theta, N, workspace=False), Yref)                  # token-major, element gather
+    check(spgemm(X, packed, theta, N, split_k=3, out_f32=True), Yref, True)
+    check(spgemm(X, packed, theta, N, channel_major=True), Yref)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=1, split_k=2), Yref)
+
+
+def test_identity_permutation_and_unit_rows():
+    """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(5, 256, 256)
+    packed = pack_on_gpu(vals, meta)
+    E = np.eye(256, dtype=np.float16)
+    Y = spgemm(E, packed, None, 256, out_f32=True)
+    assert np.array_equal(Y.astype(np.float16).view(np.uint16).T,
+                          orc.decompress_permuted(vals, meta).view(np.uint16))
+    Yp = spgemm(E, packed, theta, 256, out_f32=True)
+    assert np.array_equal(Yp.astype(np.float16).view(np.uint16).T, orc.decompress(vals, meta, theta).view(np.uint16))
+
+
+def test_split_k_is_deterministic_and_order_fixed():
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(9, 256, 2048)
+    packed = pack_on_gpu(vals, meta)
+    X = np.random.default_rng(1).standard_normal((16, 2048)).astype(np.float16)
+    a = spgemm(X, packed, theta, 256, split_k=8, out_f32=True)
+    for _ in range(3):
+        assert np.array_equal(a, spgemm(X, packed, theta, 256, split_k=8, out_f32=True))
+    check(a, orc.product(X, vals, meta, theta), True)
+
+
+def test_llama7b_shapes_sampled_outputs():
+    """Full-size config-1 GEMM shapes in the launch configuration the benchmark times; the oracle checks a
+    seeded sample of whole token rows x feature columns plus tile-boundary rows and columns."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    wl = inputs.WORKLOADS[1]
+    g = np.random.default_rng(11)
+    for (N, K), lin in inputs.distinct_shapes(wl).items():
+        W = inputs.make_weight(wl, lin)
+        s = 1.0 + g.random(K)
+        theta = g.permutation(K).astype(np.int32)
+        vals, meta, _ = orc.select_compress(W, s, theta)
+        packed = pack_on_gpu(vals, meta)
+        for M in (1, 16, 128, 2048):
+            X = inputs.make_gemm_x(wl, lin, M)
+            Y = spgemm(X, packed, theta, N)
+            rows = np.unique(np.concatenate([g.choice(M, min(M, 8), replace=False), [0, M - 1, min(M - 1, 255), min(M - 1, 256)]]))
+            cols = np.unique(np.concatenate([g.choice(N, 48, replace=False), [0, 127, 128, N - 1]]))
+            Yref = orc.product_entries(X, vals, meta, theta, rows, cols)
+            check(Y[np.ix_(rows, cols)], Yref)
