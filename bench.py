@@ -224,9 +224,13 @@ def run_ours(args):
             xs.append(X.t().contiguous() if channel_major else X)
         return xs
 
-    def gemm_step(xs, ys, opts):
+    def make_ws(M, opts):
+        n = max(b.esp_spgemm_workspace_bytes(M, lin["N"], lin["K"], opts) for lin in layer)
+        return torch.empty(n, dtype=torch.uint8, device=dev) if n else None
+
+    def gemm_step(xs, ys, opts, ws=None):
         for lin, X, Y in zip(layer, xs, ys):
-            b.esp_spgemm(X, lin["packed"], lin["perm"], Y, opts)
+            b.esp_spgemm(X, lin["packed"], lin["perm"], Y, opts, ws)
 
     results = {}
     # ---------------- prefill (headline) ----------------
@@ -239,7 +243,8 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
-    ms = time_steps(lambda: gemm_step(xs, ys, po), args.steps, args.warmup)
+    pws = make_ws(PREFILL_M, po)
+    ms = time_steps(lambda: gemm_step(xs, ys, po, pws), args.steps, args.warmup)
     clocks = sampler.stop()
     if dist:
         t = torch.tensor([ms], device=dev)
@@ -259,7 +264,7 @@ def run_ours(args):
     def e2e_step():
         for lin, H, X, Y, HY in zip(layer, hx, xs, ys, hy):
             X.copy_(H, non_blocking=True)
-            b.esp_spgemm(X, lin["packed"], lin["perm"], Y, po)
+            b.esp_spgemm(X, lin["packed"], lin["perm"], Y, po, pws)
             HY.copy_(Y, non_blocking=True)
     e2e_ms = time_steps(e2e_step, max(2, args.steps // 4), 2)
     if dist:
@@ -274,9 +279,12 @@ def run_ours(args):
     if rank == 0:
         # ---------------- decode regime: HBM-bound ----------------
         do = b.esp_gemm_opts_default()
-        dx = make_x(DECODE_M, False)
+        do.x_layout = po.x_layout
+        dx = make_x(DECODE_M, args.x_layout == "channel")
         dy = [torch.empty(DECODE_M, lin["N"], dtype=torch.float16, device=dev) for lin in layer]
-        dms = time_steps(lambda: gemm_step(dx, dy, do), max(args.steps, 50), max(args.warmup, 5))
+        dws = make_ws(DECODE_M, do)
+        dms = time_steps(lambda: gemm_step(dx, dy, do, dws), max(args.steps, 50), max(args.warmup, 5))
+        dxt = dx if args.x_layout != "channel" else make_x(DECODE_M, False)
         dbytes = sum(gemm_bytes(DECODE_M, lin["N"], lin["K"]) for lin in layer)
         dgbs = dbytes / (dms * 1e-3) / 1e9
         extra["decode"] = {"M": DECODE_M, "ms_per_step": dms, "value": dgbs, "unit": "GB/s",
@@ -289,7 +297,20 @@ def run_ours(args):
                 torch.matmul(X, lin["W"].t())
         xs_tok = xs if args.x_layout != "channel" else make_x(PREFILL_M, False)
         dense_ms = time_steps(lambda: dense_step(xs_tok), args.steps, args.warmup)
-        dense_dec_ms = time_steps(lambda: dense_step(dx), max(args.steps, 50), max(args.warmup, 5))
+        dense_dec_ms = time_steps(lambda: dense_step(dxt), max(args.steps, 50), max(args.warmup, 5))
+        # the other activation layout, for the record (token-major goes through a transposed copy of X)
+        other = "token" if args.x_layout == "channel" else "channel"
+        oo = b.esp_gemm_opts_default()
+        oo.x_layout = b.ESP_X_CHANNEL_MAJOR if other == "channel" else b.ESP_X_TOKEN_MAJOR
+        oxs = make_x(PREFILL_M, other == "channel")
+        ows = make_ws(PREFILL_M, oo)
+        oms = time_steps(lambda: gemm_step(oxs, ys, oo, ows), max(2, args.steps // 2), 3)
+        odx = make_x(DECODE_M, other == "channel")
+        odws = make_ws(DECODE_M, oo)
+        odms = time_steps(lambda: gemm_step(odx, dy, oo, odws), max(args.steps, 50), 5)
+        extra["other_x_layout"] = {"x_layout": other, "prefill_tflops": flops / (oms * 1e-3) / 1e12,
+                                   "decode_gbs": dbytes / (odms * 1e-3) / 1e9}
+        del oxs, odx
         extra["dense_cublas_f16"] = {"prefill_ms_per_step": dense_ms, "prefill_tflops": flops / (dense_ms * 1e-3) / 1e12,
                                      "decode_ms_per_step": dense_dec_ms,
                                      "speedup_prefill": dense_ms / ms, "speedup_decode": dense_dec_ms / dms}
@@ -330,18 +351,63 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_profile_case(args):
+    """A few launches of one kernel on one LLaMA-7B-shaped linear, sized for an ncu capture (tens of MB on
+    the device).  Weights are random kept values with legal metadata: traffic and timing do not depend on
+    the values.  Prints the CUDA-event time of the launches it made."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    dev = torch.device("cuda", 0)
+    torch.manual_seed(1)
+    case = args.profile_case
+    N, K = (4096, 4096)
+    if case == "prune":
+        from paper_2310_15929_b200 import inputs
+        wl = inputs.WORKLOADS[WORKLOAD]
+        T = 4096
+        W = torch.from_numpy(inputs.make_weight(wl, "q", No=1024)).to(dev)
+        Xc = torch.from_numpy(inputs.make_calibration(wl, "q", T=T)).to(dev)
+        o = b.esp_prune_opts_default(); o.alpha = 1.0 / math.sqrt(T); o.lbs_max_swaps = 2
+        ws = torch.empty(b.esp_metric_prune_workspace_bytes(1024, K, T, o), dtype=torch.uint8, device=dev)
+        vals = torch.empty(1024, K // 2, dtype=torch.float16, device=dev)
+        meta = torch.empty(1024, K // 8, dtype=torch.uint8, device=dev)
+        perm = torch.empty(K, dtype=torch.int32, device=dev)
+        packed = torch.empty(b.esp_packed_bytes(1024, K), dtype=torch.uint8, device=dev)
+        fn = lambda: b.esp_metric_prune(W, Xc, o, vals, meta, perm, packed, workspace=ws)
+        ms = time_steps(fn, 2, 1)
+        print(json.dumps({"case": case, "No": 1024, "C": K, "T": T, "ms": ms}))
+        return
+    M = PREFILL_M if case == "prefill" else DECODE_M
+    vals = (torch.randn(N, K // 2, device=dev) * 0.02).half()
+    meta = torch.full((N, K // 8), 0xE4, dtype=torch.uint8, device=dev)
+    packed = torch.empty(b.esp_packed_bytes(N, K), dtype=torch.uint8, device=dev)
+    b.esp_pack(vals, meta, N, K, packed)
+    perm = torch.randperm(K, device=dev).int()
+    X = torch.randn(K, M, device=dev).half()
+    Y = torch.empty(M, N, dtype=torch.float16, device=dev)
+    o = b.esp_gemm_opts_default(); o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    ms = time_steps(lambda: b.esp_spgemm(X, packed, perm, Y, o), 3, 3)
+    print(json.dumps({"case": case, "M": M, "N": N, "K": K, "ms_per_launch": ms,
+                      "tflops": 2.0 * M * N * K / ms / 1e9, "gbs": gemm_bytes(M, N, K) / ms / 1e6}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--x-layout", default="token", choices=["token", "channel"])
+    ap.add_argument("--x-layout", default="channel", choices=["token", "channel"],
+                    help="activation layout handed to esp_spgemm: channel = [K, M] (channels are rows)")
     ap.add_argument("--lbs-max-swaps", type=int, default=8,
                     help="cap on block-shuffle swaps per block while preparing the weights (0 = run to the end)")
     ap.add_argument("--cpu-rows", type=int, default=256)
+    ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "prune"],
+                    help="run a few launches of one small case (for ncu) instead of the benchmark")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_case:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -137,9 +137,13 @@ enum { ESP_X_TOKEN_MAJOR = 0,    /* X[t, c] at X + t * ldx + c  (tokens are rows
 enum { ESP_OUT_F16 = 0, ESP_OUT_F32 = 1 };
 enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_GATHER = 1,    /* element gather of X, any layout, no workspace (slow for large M)    */
-       ESP_KERNEL_TMA = 2,       /* channel-major X tiles fetched row-wise by the tensor memory unit    */
-       ESP_KERNEL_RESIDENT = 3 };/* small M: the CTA's whole K-slice of X is gathered once, then only
+       ESP_KERNEL_TMA = 2,       /* channel-major X rows fetched four at a time by the tensor memory
+                                    unit's row gather (correct, but that unit retires such gathers too
+                                    slowly to feed the MMA; kept for comparison)                        */
+       ESP_KERNEL_RESIDENT = 3,  /* small M: the CTA's whole K-slice of X is gathered once, then only
                                     weight tiles stream                                                 */
+       ESP_KERNEL_STREAM = 4 };  /* large M: channel-major X rows streamed by asynchronous 16-byte
+                                    copies, weight tiles by bulk copies                                 */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */

@@ -16,7 +16,7 @@ ESP_ERR_INVALID_ARG, ESP_ERR_SHAPE, ESP_ERR_ALIGNMENT, ESP_ERR_WORKSPACE = 1, 2,
 ESP_ERR_UNSUPPORTED, ESP_ERR_CUDA, ESP_ERR_TIMEOUT = 5, 6, 7
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
-ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_RESIDENT = 0, 1, 2, 3
+ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_RESIDENT, ESP_KERNEL_STREAM = 0, 1, 2, 3, 4
 
 
 class esp_prune_opts(ctypes.Structure):

@@ -41,7 +41,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->x_layout != ESP_X_TOKEN_MAJOR && o->x_layout != ESP_X_CHANNEL_MAJOR) return ESP_ERR_INVALID_ARG;
     if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
-    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_RESIDENT) return ESP_ERR_INVALID_ARG;
+    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_STREAM) return ESP_ERR_INVALID_ARG;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
 }

@@ -11,6 +11,8 @@
 // distributed shared memory, so no global scratch is used and the result is deterministic.
 #include "esp_common.cuh"
 
+#include <cuda.h>
+
 namespace esp {
 namespace {
 
@@ -558,6 +560,466 @@ __global__ void __launch_bounds__(192) spgemm_resident_kernel(const GemmParams p
     }
 }
 
+
+// --------------------------------------------------------------------------------------------------
+// TMA kernel: large token counts (prefill), channel-major X.
+// The X tile of a stage is 128 permuted channels x BN tokens.  Channel rows are fetched by the tensor
+// memory unit four arbitrary rows at a time (tile::gather4, row indices = 4 consecutive entries of the
+// permutation), 64 tokens (128 bytes) per row, landing 128-byte swizzled as an MN-major B operand: the
+// permutation costs nothing beyond the loads themselves and no permuted copy of X exists anywhere.
+// grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192:
+//   warp 0  producer: lane 0 issues the weight-tile bulk copy, all lanes issue gather4 row loads
+//   warp 1  lane 0 issues tcgen05.cp (metadata) + 4 sparse MMAs per stage
+//   warps 2..5  epilogue
+// --------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int x, int r0, int r1, int r2, int r3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+        : "memory");
+}
+
+template <int BN>
+struct TmaCfg {
+    static constexpr int kXStage = 128 * BN * 2;
+    static constexpr int kStage = kTileBytes + kXStage;
+    static constexpr int kStages = (BN == 256) ? 2 : (BN == 128) ? 4 : 6;
+    static constexpr int kBarOff = kStages * kStage;
+    static constexpr int kTotal = kBarOff + 256 + 1024;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap xmap) {
+    using L = TmaCfg<BN>;
+    constexpr int STAGES = L::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + L::kBarOff;
+    auto full = [&](int s) { return bar_base + 8u * s; };
+    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
+    const uint32_t accum_bar = bar_base + 8u * 16;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 17);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 17 + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
+    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
+    const int kt_begin = slice * p.k_tiles_per_split;
+    const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
+    const int nk = max(0, kt_end - kt_begin);
+    constexpr uint32_t kTmemCols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
+        bool alive = true;
+        for (int it = 0; it < nk && alive; ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+            // this lane's permutation entries: rows 4*lane .. 4*lane+3 of the stage
+            const int kpos = (kt_begin + it) * kTileK + lane * 4;
+            int4 rows;
+            if (kpos + 4 <= p.K && p.perm) {
+                rows = __ldg(reinterpret_cast<const int4 *>(p.perm + kpos));
+            } else {
+                int r[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) r[e] = (kpos + e < p.K) ? (p.perm ? __ldg(p.perm + kpos + e) : kpos + e) : p.K;   // K = out of range: zero fill
+                rows = make_int4(r[0], r[1], r[2], r[3]);
+            }
+            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { alive = false; }
+            alive = __all_sync(0xFFFFFFFFu, alive);
+            if (!alive) break;
+            const uint32_t stage = sbase + s * L::kStage;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(full(s), L::kStage);
+                bulk_load(stage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
+            }
+            __syncwarp();
+#pragma unroll
+            for (int tb = 0; tb < BN / 64; ++tb)
+                tma_gather4(stage + kTileBytes + tb * 16384 + lane * 512, &xmap, tok0 + tb * 64, rows.x, rows.y, rows.z, rows.w, full(s));
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(full(s), ph, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t wa = sbase + s * L::kStage;
+                const uint32_t xa = wa + kTileBytes;
+                const uint32_t e_col = BN + (it & 1) * 4;
+                tc_copy_128x128b(tmem + e_col, smem_desc(wa + kTileValBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t col = e_col + j;
+                    const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
+                    const uint64_t bd = smem_desc(xa + j * 4096, 16384, 1024, kLayoutSw128);
+                    tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            tc_commit(accum_bar);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int f_local = quarter * 32 + lane;
+        const long feature = (long)ft * 128 + f_local;
+        const bool ok = (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
+        tc_fence_after();
+        float *stage_f32 = reinterpret_cast<float *>(smem);
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+            uint32_t v[16];
+            if (nk > 0) {
+                tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0;
+            }
+            if (split == 1) {
+                if (ok && feature < p.N) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int t = tok0 + c0 + e;
+                        if (t < p.M) {
+                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
+                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
+                        }
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+            }
+        }
+        tc_fence_before();
+    }
+
+    if (split > 1) {
+        cluster_sync_all();
+        const uint32_t rank = cluster_ctarank();
+        const bool ok = (*abort_flag == 0);
+        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
+            const int row = idx >> 7, f_local = idx & 127;
+            if ((row % split) != (int)rank) continue;
+            const int t = tok0 + row;
+            const long feature = (long)ft * 128 + f_local;
+            if (t >= p.M || feature >= p.N) continue;
+            float acc = 0.f;
+            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
+            if (ok) {
+                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
+                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
+            }
+        }
+        cluster_sync_all();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+
+// --------------------------------------------------------------------------------------------------
+// Streaming kernel: large token counts (prefill), channel-major X.  Same tiles and operand layouts as the
+// row-gather kernel above, but the 128 permuted channel rows of a stage are fetched by four producer
+// warps with 16-byte asynchronous copies (cp.async), 8 lanes per 128-byte row segment, which complete on
+// the stage's mbarrier.  (Measured on B200: the tensor memory unit retires one four-row gather per ~60
+// clocks, 8.5 B/clk per SM, far below what the MMA consumes; plain asynchronous row copies are not bound
+// by that.)  The epilogue transposes the accumulator tile through shared memory so that Y is written in
+// full 16-byte pieces along the feature dimension.
+// grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192:
+//   warp 0 lane 0  weight-tile producer (bulk async copy)     warp 1 lane 0  tcgen05.cp + sparse MMAs
+//   warps 2..5     X row producers, then epilogue
+// --------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int BN>
+__global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams p) {
+    using L = TmaCfg<BN>;
+    constexpr int STAGES = L::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + L::kBarOff;
+    auto full = [&](int s) { return bar_base + 8u * s; };
+    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
+    const uint32_t accum_bar = bar_base + 8u * 16;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 17);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 17 + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
+    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
+    const int kt_begin = slice * p.k_tiles_per_split;
+    const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
+    const int nk = max(0, kt_end - kt_begin);
+    constexpr uint32_t kTmemCols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 128 + 1); mbar_init(empty(s), 1); }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(full(s), kTileBytes);
+                bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(full(s), ph, abort_flag)) break;
+                fence_async_smem();          // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
+                tc_fence_after();
+                const uint32_t wa = sbase + s * L::kStage;
+                const uint32_t xa = wa + kTileBytes;
+                const uint32_t e_col = BN + (it & 1) * 4;
+                tc_copy_128x128b(tmem + e_col, smem_desc(wa + kTileValBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t col = e_col + j;
+                    const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
+                    const uint64_t bd = smem_desc(xa + j * 4096, 16384, 1024, kLayoutSw128);
+                    tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            tc_commit(accum_bar);
+        }
+    } else {
+        // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) + 16 i of every 64-token block
+        const int g = threadIdx.x - 64;
+        const int cc = g & 7, rg = g >> 3;
+        const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
+        bool alive = true;
+        for (int it = 0; it < nk; ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+            int ch[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int kpos = (kt_begin + it) * kTileK + rg + 16 * i;
+                ch[i] = (kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+            }
+            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+            const uint32_t xs = sbase + s * L::kStage + kTileBytes;
+#pragma unroll
+            for (int tb = 0; tb < BN / 64; ++tb) {
+                const int t = tok0 + tb * 64 + cc * 8;
+                const int valid = min(8, max(0, p.M - t));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = rg + 16 * i;
+                    const bool in = ch[i] >= 0 && valid > 0;
+                    const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
+                    cp_async_16(xs + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4), src, in ? valid * 2 : 0);
+                }
+            }
+            cp_async_arrive_noinc(full(s));
+        }
+        // ---- epilogue
+        const int quarter = warp & 3;
+        const int f_local = quarter * 32 + lane;
+        const bool ok = alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
+        tc_fence_after();
+        if (split == 1) {
+            // accumulators -> shared memory [token][128 features] in the output type -> 16-byte stores
+            const int esize = p.out_f32 ? 4 : 2;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t v[16];
+                if (nk > 0) {
+                    tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0;
+                }
+                if (p.out_f32) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
+                }
+            }
+            tc_fence_before();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int row_bytes = 128 * esize;
+            const int chunks_per_row = row_bytes / 16;
+            const int f_valid = min(128, p.N - ft * 128);
+            const bool vec_ok = (((long)p.ldy * esize) % 16 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0);
+            uint8_t *yb = reinterpret_cast<uint8_t *>(p.Y);
+            for (int idx = g; idx < BN * chunks_per_row; idx += 128) {
+                const int row = idx / chunks_per_row, c = idx % chunks_per_row;
+                const int t = tok0 + row;
+                if (!ok || t >= p.M) continue;
+                const int f0 = c * (16 / esize);
+                uint8_t *dst = yb + ((long)t * p.ldy + (long)ft * 128 + f0) * esize;
+                const uint8_t *srcp = smem + (size_t)row * row_bytes + c * 16;
+                if (vec_ok && f0 + 16 / esize <= f_valid) {
+                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(srcp);
+                } else {
+                    for (int e = 0; e < 16 / esize; ++e)
+                        if (f0 + e < f_valid) {
+                            if (p.out_f32) reinterpret_cast<float *>(dst)[e] = reinterpret_cast<const float *>(srcp)[e];
+                            else reinterpret_cast<uint16_t *>(dst)[e] = reinterpret_cast<const uint16_t *>(srcp)[e];
+                        }
+                }
+            }
+        } else {
+            float *stage_f32 = reinterpret_cast<float *>(smem);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t v[16];
+                if (nk > 0) {
+                    tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0;
+                }
+#pragma unroll
+                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+            }
+            tc_fence_before();
+        }
+    }
+
+    if (split > 1) {
+        cluster_sync_all();
+        const uint32_t rank = cluster_ctarank();
+        const bool ok = (*abort_flag == 0);
+        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
+            const int row = idx >> 7, f_local = idx & 127;
+            if ((row % split) != (int)rank) continue;
+            const int t = tok0 + row;
+            const long feature = (long)ft * 128 + f_local;
+            if (t >= p.M || feature >= p.N) continue;
+            float acc = 0.f;
+            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
+            if (ok) {
+                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
+                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
+            }
+        }
+        cluster_sync_all();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+template <int BN>
+esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int split, cudaStream_t stream) {
+    using L = TmaCfg<BN>;
+    auto kern = spgemm_stream_kernel<BN>;
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(f_tiles, t_tiles, split);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
+    return ESP_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map over channel-major X: dim 0 = tokens (contiguous), dim 1 = channels (ldx apart); box = 64 tokens
+// x 1 row (the row-gather form loads four such rows per instruction), 128-byte swizzle, zero fill outside.
+inline esp_status_t make_x_tensor_map(const __half *X, int M, int K, long ldx, CUtensorMap *map) {
+    static EncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+            return ESP_ERR_CUDA;
+        encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)K};
+    cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
+    cuuint32_t box[2] = {64, 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half *>(X), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? ESP_OK : ESP_ERR_CUDA;
+}
+
+template <int BN>
+esp_status_t launch_tma(const GemmParams &p, int f_tiles, int t_tiles, int split, cudaStream_t stream) {
+    using L = TmaCfg<BN>;
+    CUtensorMap map;
+    esp_status_t st = make_x_tensor_map(p.X, p.M, p.K, p.ldx, &map);
+    if (st != ESP_OK) return st;
+    auto kern = spgemm_tma_kernel<BN>;
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(f_tiles, t_tiles, split);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, map));
+    return ESP_OK;
+}
+
 inline size_t resident_smem_bytes(int bn, int stages, int k_tiles_per_split) {
     return (size_t)stages * kTileBytes + (size_t)k_tiles_per_split * 128 * bn * 2 + 256 + 1024;
 }
@@ -621,9 +1083,17 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
     const bool channel_major_available = (o.x_layout == ESP_X_CHANNEL_MAJOR) || have_workspace;
     int bn = o.token_tile;
     g.kernel = ESP_KERNEL_GATHER;
-    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available && M <= 64 && (bn == 0 || bn <= 64))
-        g.kernel = ESP_KERNEL_RESIDENT;
+    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available) {
+        const bool small = M <= 64 && (bn == 0 || bn <= 64);
+        if (o.force_kernel == ESP_KERNEL_RESIDENT) g.kernel = small ? ESP_KERNEL_RESIDENT : ESP_KERNEL_GATHER;
+        else if (o.force_kernel == ESP_KERNEL_TMA) g.kernel = ESP_KERNEL_TMA;
+        else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
+        else g.kernel = small ? ESP_KERNEL_RESIDENT : ESP_KERNEL_STREAM;
+    }
+    const bool tiled = (g.kernel == ESP_KERNEL_TMA || g.kernel == ESP_KERNEL_STREAM);
+    if (tiled && bn != 0 && bn < 64) bn = 64;
     if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    if (tiled && bn < 64) bn = 64;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
     const int t_tiles = ceil_div(M, bn);
@@ -641,7 +1111,7 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
         if (split < min_split) split = min_split;
         if ((size_t)ceil_div(k_tiles, split) * 128 * bn * 2 > 96 * 1024) g.kernel = ESP_KERNEL_GATHER;
     }
-    if (g.kernel == ESP_KERNEL_GATHER && split == 0) {
+    if (g.kernel != ESP_KERNEL_RESIDENT && split == 0) {
         split = 1;
         while (split < 8 && (long)f_tiles * t_tiles * split < di.sm_count && k_tiles / (split * 2) >= 4) split *= 2;
     }
@@ -675,7 +1145,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.k_tiles = ceil_div(K, kTileK);
     p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
-    if (plan.kernel == ESP_KERNEL_RESIDENT) {
+    if (plan.kernel != ESP_KERNEL_GATHER) {
         if (!p.x_channel_major) {
             // token-major input: transposed (not permuted) copy into the caller's workspace
             const long ldt = transposed_ld(M);
@@ -686,6 +1156,22 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.X = reinterpret_cast<const __half *>(workspace);
             p.ldx = ldt;
             p.x_channel_major = 1;
+        }
+        if (plan.kernel == ESP_KERNEL_STREAM) {
+            switch (plan.token_tile) {
+                case 64: return launch_stream<64>(p, f_tiles, t_tiles, plan.split_k, stream);
+                case 128: return launch_stream<128>(p, f_tiles, t_tiles, plan.split_k, stream);
+                case 256: return launch_stream<256>(p, f_tiles, t_tiles, plan.split_k, stream);
+                default: return ESP_ERR_INVALID_ARG;
+            }
+        }
+        if (plan.kernel == ESP_KERNEL_TMA) {
+            switch (plan.token_tile) {
+                case 64: return launch_tma<64>(p, f_tiles, t_tiles, plan.split_k, stream);
+                case 128: return launch_tma<128>(p, f_tiles, t_tiles, plan.split_k, stream);
+                case 256: return launch_tma<256>(p, f_tiles, t_tiles, plan.split_k, stream);
+                default: return ESP_ERR_INVALID_ARG;
+            }
         }
         switch (plan.token_tile) {
             case 16: return launch_resident<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);

@@ -72,6 +72,26 @@ def test_decode_and_ragged_shapes(M, N, K):
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=1, split_k=2), Yref)
 
 
+@pytest.mark.parametrize("kernel", [4, 2])
+@pytest.mark.parametrize("M", [65, 130, 300, 520])
+@pytest.mark.parametrize("N,K", [(256, 512), (200, 264), (384, 1160)])
+def test_prefill_tiled_kernels(M, N, K, kernel):
+    """Large-M kernels (4 = asynchronous row copies, 2 = tensor-memory-unit row gather): ragged token /
+    feature / channel tails, K-slices, both activation layouts, both output types."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(N * 3 + K + M, N, K)
+    X = np.random.default_rng(M + 1).standard_normal((M, K)).astype(np.float16)
+    Yref = orc.product(X, vals, meta, theta)
+    packed = pack_on_gpu(vals, meta)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel), Yref)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel, out_f32=True), Yref, True)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel, token_tile=64, split_k=2, out_f32=True), Yref, True)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel, token_tile=128), Yref)
+    check(spgemm(X, packed, theta, N, kernel=kernel), Yref)                     # token-major via the transposed copy
+    check(spgemm(X, packed, None, N, channel_major=True, kernel=kernel),
+          orc.product(X, vals, meta, None))
+
+
 def test_identity_permutation_and_unit_rows():
     """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
     from tests.gpu_util import pack_on_gpu, spgemm
