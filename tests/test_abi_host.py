@@ -51,7 +51,10 @@ def test_size_queries():
     big = b.esp_metric_prune_workspace_bytes(4096, 4096, 32768, o)
     assert 0 < small < big
     assert b.esp_metric_prune_workspace_bytes(512, 510, 128, o) == 0           # C % 8 != 0
-    assert b.esp_spgemm_workspace_bytes(16, 4096, 4096, b.esp_gemm_opts_default()) == 0
+    g = b.esp_gemm_opts_default()
+    assert b.esp_spgemm_workspace_bytes(16, 4096, 4096, g) == 4096 * 16 * 2     # transposed copy of token-major X
+    g.x_layout = b.ESP_X_CHANNEL_MAJOR
+    assert b.esp_spgemm_workspace_bytes(16, 4096, 4096, g) == 0                 # K-slices reduce on chip: no scratch
 
 
 A = 0x10000   # a fake, 16-byte aligned "device address": argument errors must be caught before any use
