@@ -40,7 +40,8 @@ typedef enum {
     ESP_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than the *_workspace_bytes() answer       */
     ESP_ERR_UNSUPPORTED = 5,   /* pattern other than 2:4, bins > 1024, device is not sm_100           */
     ESP_ERR_CUDA = 6,          /* a CUDA runtime call or a launch failed                              */
-    ESP_ERR_TIMEOUT = 7        /* a bounded in-kernel wait gave up (reported by esp_last_device_status) */
+    ESP_ERR_TIMEOUT = 7,       /* a bounded in-kernel wait gave up (reported by esp_last_device_status) */
+    ESP_ERR_STATIC_LIMIT = 8   /* esp_spgemm_static: the sizes need more than ESP_STATIC_SCRATCH_BYTES   */
 } esp_status_t;
 
 /* Static string for a status code (never NULL). */
@@ -178,6 +179,33 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx,
                         const void *packed, const int32_t *perm, int N,
                         void *Y, long ldy, const esp_gemm_opts *opts,
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The product for hosts that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * deployment convenience of this library, not a step of the method.)
+ *
+ * Same result as esp_spgemm with token-major X (X[t, c] at X + t * ldx + c), default options and a
+ * workspace -- but the transposed copy of X that the fast kernels read goes into a fixed array of
+ * ESP_STATIC_SCRATCH_BYTES inside the library's device image, so the caller passes only inputs and outputs
+ * and the call performs no cudaMalloc, cudaFree or other allocation.  It is meant for callers that run
+ * layers from a hook which carries no workspace pointer while all device memory belongs to their host
+ * engine's pool, and for threads that must not call cudaMalloc because it can synchronise the device.
+ *
+ *   - Limit: K * round_up(M, 16) * 2 bytes must not exceed ESP_STATIC_SCRATCH_BYTES (8 MiB: M <= 1024 at
+ *     K = 4096, M <= 112 at K = 36864); larger sizes return ESP_ERR_STATIC_LIMIT and launch nothing.
+ *     Every GPU on which the library is loaded holds the array until the process exits.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Nothing in it
+ *     has to start at zero (the region a call reads is rewritten in full first), but two calls whose
+ *     kernels overlap on the GPU -- different streams, or the same call from two threads -- race on it:
+ *     keep calls to this entry point stream-ordered with respect to each other.
+ *   - out_dtype is ESP_OUT_F16 or ESP_OUT_F32; perm NULL = identity; other arguments as in esp_spgemm.
+ */
+#define ESP_STATIC_SCRATCH_BYTES (8u << 20)
+esp_status_t esp_spgemm_static(const void *X, int M, int K, long ldx,
+                               const void *packed, const int32_t *perm, int N,
+                               void *Y, long ldy, int out_dtype, void *cuda_stream);
 
 /*
  * Reads and clears the device-side status word of the current device (synchronises the device).

@@ -14,6 +14,8 @@ from .build import LIB_PATH
 ESP_OK = 0
 ESP_ERR_INVALID_ARG, ESP_ERR_SHAPE, ESP_ERR_ALIGNMENT, ESP_ERR_WORKSPACE = 1, 2, 3, 4
 ESP_ERR_UNSUPPORTED, ESP_ERR_CUDA, ESP_ERR_TIMEOUT = 5, 6, 7
+ESP_ERR_STATIC_LIMIT = 8
+ESP_STATIC_SCRATCH_BYTES = 8 << 20
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
 ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_RESIDENT, ESP_KERNEL_STREAM = 0, 1, 2, 3, 4
@@ -48,7 +50,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_gemm_opts_default",
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
-           "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status")
+           "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
+           "esp_spgemm_static")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -73,6 +76,9 @@ _lib.esp_spgemm.restype = c_int
 _lib.esp_spgemm.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
                             POINTER(esp_gemm_opts), c_void_p, c_size_t, c_void_p]
 _lib.esp_last_device_status.restype = c_int
+_lib.esp_spgemm_static.restype = c_int
+_lib.esp_spgemm_static.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
+                                   c_int, c_void_p]
 
 
 def _ptr(t):
@@ -180,6 +186,23 @@ def esp_spgemm(X, packed, perm, Y, opts, workspace=None, stream=None):
                         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
     if st != ESP_OK:
         raise EsparseError(st, "esp_spgemm")
+
+
+def esp_spgemm_static_raw(X, M, K, ldx, packed, perm, N, Y, ldy, out_dtype, stream) -> int:
+    return int(_lib.esp_spgemm_static(_ptr(X), M, K, ldx, _ptr(packed), _ptr(perm), N, _ptr(Y), ldy, out_dtype,
+                                      stream))
+
+
+def esp_spgemm_static(X, packed, perm, Y, stream=None):
+    """Y [M,N] = X . P . W_s^T for token-major X [M,K] with the library's built-in scratch: no workspace and
+    no allocation (for callers that cannot allocate device memory).  Y's dtype picks fp16 or fp32 output."""
+    import torch
+    M, N = Y.shape
+    K = X.shape[1]
+    out = ESP_OUT_F32 if Y.dtype == torch.float32 else ESP_OUT_F16
+    st = esp_spgemm_static_raw(X, M, K, X.stride(0), packed, perm, N, Y, Y.stride(0), out, _stream(stream))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_spgemm_static")
 
 
 def esp_last_device_status() -> int:

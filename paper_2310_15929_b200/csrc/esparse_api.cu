@@ -62,6 +62,7 @@ const char *esp_status_string(esp_status_t status) {
         case ESP_ERR_UNSUPPORTED: return "unsupported configuration or device";
         case ESP_ERR_CUDA: return "CUDA runtime error";
         case ESP_ERR_TIMEOUT: return "a bounded in-kernel wait gave up";
+        case ESP_ERR_STATIC_LIMIT: return "sizes exceed the built-in scratch of esp_spgemm_static";
         default: return "unknown status";
     }
 }

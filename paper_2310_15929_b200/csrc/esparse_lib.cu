@@ -2,3 +2,4 @@
 #include "prune_kernels.cu"
 #include "spgemm_kernels.cu"
 #include "esparse_api.cu"
+#include "spgemm_static.cu"
