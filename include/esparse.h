@@ -141,10 +141,8 @@ enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_TMA = 2,       /* channel-major X rows fetched four at a time by the tensor memory
                                     unit's row gather (correct, but that unit retires such gathers too
                                     slowly to feed the MMA; kept for comparison)                        */
-       ESP_KERNEL_RESIDENT = 3,  /* small M: the CTA's whole K-slice of X is gathered once, then only
-                                    weight tiles stream                                                 */
-       ESP_KERNEL_STREAM = 4 };  /* large M: channel-major X rows streamed by asynchronous 16-byte
-                                    copies, weight tiles by bulk copies                                 */
+       ESP_KERNEL_STREAM = 4 };  /* channel-major X rows streamed by asynchronous 16-byte copies, weight
+                                    tiles by bulk copies; every token count (the default)               */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
@@ -152,7 +150,12 @@ typedef struct {
     int out_dtype;               /* ESP_OUT_*: type of Y                                              */
     int split_k;                 /* K-slices reduced inside a thread-block cluster; 0 = choose, 1..8  */
     int force_kernel;            /* ESP_KERNEL_*                                                      */
-    int token_tile;              /* tokens per CTA tile (16..256, multiple of 16); 0 = choose         */
+    int token_tile;              /* tokens per CTA tile (16, 32, 64, 128 or 256); 0 = choose          */
+    int static_weights;          /* 1 = `packed` and `perm` are not written by work still pending on the
+                                    stream (the usual case at inference).  The kernel is then launched as
+                                    a programmatic dependent of the preceding kernel: its weight prefetch
+                                    overlaps that kernel's tail, and only the reads of X and the writes
+                                    of Y wait for it.  0 (default) = plain stream order.                 */
 } esp_gemm_opts;
 
 void esp_gemm_opts_default(esp_gemm_opts *opts);
@@ -163,6 +166,16 @@ void esp_gemm_opts_default(esp_gemm_opts *opts);
  * or smaller workspace the call still works through the element-gather kernel.
  */
 size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts);
+
+/*
+ * Reports the launch configuration esp_spgemm would use for these sizes on the current device (the
+ * counterpart of step (2) of "Efficient Sparse-GEMM Implementation", where the paper searches the library's
+ * algorithms per weight shape): kernel (ESP_KERNEL_*), tokens per CTA tile, K-slices per cluster, pipeline
+ * stages.  have_workspace says whether a workspace of esp_spgemm_workspace_bytes() will be passed.
+ * Output pointers may be NULL.  Launches nothing.
+ */
+esp_status_t esp_spgemm_plan(int M, int N, int K, const esp_gemm_opts *opts, int have_workspace,
+                             int *kernel, int *token_tile, int *split_k, int *stages);
 
 /*
  * Y[t, j] = sum over kept weights of row j:  w * X[t, perm[position of w]]   (fp32 accumulation)

@@ -18,7 +18,7 @@ ESP_ERR_STATIC_LIMIT = 8
 ESP_STATIC_SCRATCH_BYTES = 8 << 20
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
-ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_RESIDENT, ESP_KERNEL_STREAM = 0, 1, 2, 3, 4
+ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM = 0, 1, 2, 4
 
 
 class esp_prune_opts(ctypes.Structure):
@@ -34,7 +34,7 @@ class esp_prune_stats(ctypes.Structure):
 
 class esp_gemm_opts(ctypes.Structure):
     _fields_ = [("struct_size", c_size_t), ("x_layout", c_int), ("out_dtype", c_int), ("split_k", c_int),
-                ("force_kernel", c_int), ("token_tile", c_int)]
+                ("force_kernel", c_int), ("token_tile", c_int), ("static_weights", c_int)]
 
 
 class EsparseError(RuntimeError):
@@ -51,7 +51,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_gemm_opts_default",
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
-           "esp_spgemm_static")
+           "esp_spgemm_static", "esp_spgemm_plan")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -76,6 +76,9 @@ _lib.esp_spgemm.restype = c_int
 _lib.esp_spgemm.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
                             POINTER(esp_gemm_opts), c_void_p, c_size_t, c_void_p]
 _lib.esp_last_device_status.restype = c_int
+_lib.esp_spgemm_plan.restype = c_int
+_lib.esp_spgemm_plan.argtypes = [c_int, c_int, c_int, POINTER(esp_gemm_opts), c_int, POINTER(c_int), POINTER(c_int),
+                                 POINTER(c_int), POINTER(c_int)]
 _lib.esp_spgemm_static.restype = c_int
 _lib.esp_spgemm_static.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
                                    c_int, c_void_p]
@@ -169,6 +172,16 @@ def esp_spgemm_workspace_bytes(M: int, N: int, K: int, opts: esp_gemm_opts) -> i
     return int(_lib.esp_spgemm_workspace_bytes(M, N, K, ctypes.byref(opts)))
 
 
+def esp_spgemm_plan(M: int, N: int, K: int, opts: esp_gemm_opts, have_workspace: bool = True) -> dict:
+    """The launch configuration esp_spgemm would use (needs the device; launches nothing)."""
+    k, t, s, g = c_int(), c_int(), c_int(), c_int()
+    st = int(_lib.esp_spgemm_plan(M, N, K, ctypes.byref(opts), 1 if have_workspace else 0, ctypes.byref(k),
+                                  ctypes.byref(t), ctypes.byref(s), ctypes.byref(g)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_spgemm_plan")
+    return {"kernel": k.value, "token_tile": t.value, "split_k": s.value, "stages": g.value}
+
+
 def esp_spgemm_raw(X, M, K, ldx, packed, perm, N, Y, ldy, opts, workspace, workspace_bytes, stream) -> int:
     return int(_lib.esp_spgemm(_ptr(X), M, K, ldx, _ptr(packed), _ptr(perm), N, _ptr(Y), ldy,
                                ctypes.byref(opts) if opts is not None else None, _ptr(workspace), workspace_bytes,
@@ -202,7 +215,7 @@ def esp_spgemm_static(X, packed, perm, Y, stream=None):
     out = ESP_OUT_F32 if Y.dtype == torch.float32 else ESP_OUT_F16
     st = esp_spgemm_static_raw(X, M, K, X.stride(0), packed, perm, N, Y, Y.stride(0), out, _stream(stream))
     if st != ESP_OK:
-        raise EsparseError(st, "esp_spgemm_static")
+        raise EsparseError(st, "esp_spgemm_static", "esp_spgemm_plan")
 
 
 def esp_last_device_status() -> int:

@@ -41,7 +41,10 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->x_layout != ESP_X_TOKEN_MAJOR && o->x_layout != ESP_X_CHANNEL_MAJOR) return ESP_ERR_INVALID_ARG;
     if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
-    if (o->force_kernel < ESP_KERNEL_AUTO || o->force_kernel > ESP_KERNEL_STREAM) return ESP_ERR_INVALID_ARG;
+    if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
+        o->force_kernel != ESP_KERNEL_STREAM)
+        return ESP_ERR_INVALID_ARG;
+    if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
 }
@@ -93,6 +96,7 @@ void esp_gemm_opts_default(esp_gemm_opts *o) {
     o->split_k = 0;
     o->force_kernel = ESP_KERNEL_AUTO;
     o->token_tile = 0;
+    o->static_weights = 0;
 }
 
 size_t esp_metric_prune_workspace_bytes(int No, int C, int T, const esp_prune_opts *opts) {
@@ -152,6 +156,25 @@ size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts
     // K-slices are reduced through distributed shared memory inside a cluster: no global scratch for that.
     // Token-major X is first transposed (not permuted) into the workspace so channels become rows.
     return gemm_workspace_bytes(M, K, *opts);
+}
+
+esp_status_t esp_spgemm_plan(int M, int N, int K, const esp_gemm_opts *opts, int have_workspace, int *kernel,
+                             int *token_tile, int *split_k, int *stages) {
+    esp_status_t st = check_gemm_opts(opts);
+    if (st != ESP_OK) return st;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 8 != 0) return ESP_ERR_SHAPE;
+    DeviceInfo di;
+    st = device_info(&di);
+    if (st != ESP_OK) return st;
+    if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
+    GemmPlan plan;
+    st = plan_gemm(M, N, K, *opts, have_workspace != 0, &plan);
+    if (st != ESP_OK) return st;
+    if (kernel) *kernel = plan.kernel;
+    if (token_tile) *token_tile = plan.token_tile;
+    if (split_k) *split_k = plan.split_k;
+    if (stages) *stages = plan.stages;
+    return ESP_OK;
 }
 
 esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,

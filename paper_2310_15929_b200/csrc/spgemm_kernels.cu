@@ -13,6 +13,9 @@
 
 #include <cuda.h>
 
+#include <map>
+#include <mutex>
+
 namespace esp {
 namespace {
 
@@ -375,193 +378,6 @@ esp_status_t launch_gather(const GemmParams &p, int f_tiles, int t_tiles, int sp
 
 
 // --------------------------------------------------------------------------------------------------
-// Resident-X kernel: small token counts (decode), channel-major X.
-// Each CTA owns a feature tile and a K-slice.  Its whole slice of permuted X (BN tokens per channel, one
-// swizzled shared-memory row per channel: an MN-major B operand) is gathered once at start-up by all
-// threads with 16-byte loads -- one or two sectors per channel, all loads independent -- while the first
-// weight tiles are already in flight; afterwards the main loop only streams compressed weight tiles
-// (one 18 KB bulk copy per stage), which is the HBM-bound part.
-// grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192.
-// --------------------------------------------------------------------------------------------------
-template <int BN>
-__global__ void __launch_bounds__(192) spgemm_resident_kernel(const GemmParams p, const int stages) {
-    constexpr int RB = BN * 2;                       // bytes of one channel row of the X tile
-    constexpr int kXTile = 128 * RB;                 // one 128-channel tile of X
-    constexpr uint32_t kLayout = (BN == 16) ? 6u : (BN == 32) ? 4u : 2u;   // 32 / 64 / 128-byte swizzle
-    constexpr int kSwzShift = (BN == 16) ? 2 : (BN == 32) ? 1 : 0;         // row bits that feed the XOR
-    constexpr int kChunks = RB / 16;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t sbase = smem_u32(smem);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
-    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
-    const int kt_begin = slice * p.k_tiles_per_split;
-    const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
-    const int nk = max(0, kt_end - kt_begin);
-
-    const uint32_t w_base = sbase;                                   // stages x 18432
-    const uint32_t x_base = sbase + (uint32_t)stages * kTileBytes;   // k_tiles_per_split x kXTile
-    const uint32_t bar_base = x_base + (uint32_t)p.k_tiles_per_split * kXTile;
-    uint8_t *bar_ptr = smem + (size_t)stages * kTileBytes + (size_t)p.k_tiles_per_split * kXTile;
-    auto full_w = [&](int s) { return bar_base + 8u * s; };
-    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
-    const uint32_t accum_bar = bar_base + 8u * 16;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_ptr + 8 * 17);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_ptr + 8 * 17 + 4);
-    constexpr uint32_t kTmemCols = tmem_cols_for(BN);
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(full_w(s), 1); mbar_init(empty(s), 1); }
-        mbar_init(accum_bar, 1);
-        *abort_flag = 0;
-        fence_barrier_init();
-    }
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
-
-    // first weight tiles go out before the X gather so the two latencies overlap
-    const int prefetch = min(stages, nk);
-    if (threadIdx.x == 0) {
-        for (int it = 0; it < prefetch; ++it) {
-            mbar_arrive_expect_tx(full_w(it), kTileBytes);
-            bulk_load(w_base + it * kTileBytes, w_src + (long)it * kTileBytes, kTileBytes, full_w(it));
-        }
-    }
-    // gather the K-slice of X: one channel row per iteration per thread
-    {
-        const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
-        for (int r = threadIdx.x; r < nk * 128; r += 192) {
-            const int kpos = kt_begin * kTileK + r;
-            int ch = -1;
-            if (kpos < p.K) ch = p.perm ? __ldg(p.perm + kpos) : kpos;
-            uint8_t *row = smem + (size_t)stages * kTileBytes + (size_t)r * RB;
-            const int rr = r & 127;
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                const int t = tok0 + c * 8;
-                if (ch >= 0) {
-                    const uint16_t *src = xb + (long)ch * p.ldx + t;
-                    if (t + 8 <= p.M) {
-                        v = __ldg(reinterpret_cast<const uint4 *>(src));
-                    } else if (t < p.M) {
-                        uint16_t h[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) h[e] = (t + e < p.M) ? __ldg(src + e) : (uint16_t)0;
-                        v.x = h[0] | ((uint32_t)h[1] << 16); v.y = h[2] | ((uint32_t)h[3] << 16);
-                        v.z = h[4] | ((uint32_t)h[5] << 16); v.w = h[6] | ((uint32_t)h[7] << 16);
-                    }
-                }
-                const int cs = c ^ ((rr >> kSwzShift) & (kChunks - 1));
-                *reinterpret_cast<uint4 *>(row + cs * 16) = v;
-            }
-        }
-        fence_async_smem();
-    }
-    __syncthreads();
-
-    if (warp == 0) {
-        if (lane == 0) {
-            for (int it = prefetch; it < nk; ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
-                mbar_arrive_expect_tx(full_w(s), kTileBytes);
-                bulk_load(w_base + s * kTileBytes, w_src + (long)it * kTileBytes, kTileBytes, full_w(s));
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
-            for (int it = 0; it < nk; ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
-                if (!mbar_wait(full_w(s), ph, abort_flag)) break;
-                tc_fence_after();
-                const uint32_t wa = w_base + s * kTileBytes;
-                const uint32_t xa = x_base + it * kXTile;
-                const uint32_t e_col = BN + (it & 1) * 4;
-                tc_copy_128x128b(tmem + e_col, smem_desc(wa + kTileValBytes, 0, 128, kLayoutNone));
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t col = e_col + j;
-                    const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
-                    const uint64_t bd = smem_desc(xa + j * 32 * RB, 8 * RB, 8 * RB, kLayout);
-                    tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
-                }
-                tc_commit(empty(s));
-            }
-            tc_commit(accum_bar);
-        }
-    } else {
-        const int quarter = warp & 3;
-        const int f_local = quarter * 32 + lane;
-        const long feature = (long)ft * 128 + f_local;
-        const bool ok = (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
-        tc_fence_after();
-        float *stage_f32 = reinterpret_cast<float *>(smem);
-#pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 16) {
-            uint32_t v[16];
-            if (nk > 0) {
-                tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = 0;
-            }
-            if (split == 1) {
-                if (ok && feature < p.N) {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int t = tok0 + c0 + e;
-                        if (t < p.M) {
-                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
-                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
-                        }
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
-            }
-        }
-        tc_fence_before();
-    }
-
-    if (split > 1) {
-        cluster_sync_all();
-        const uint32_t rank = cluster_ctarank();
-        const bool ok = (*abort_flag == 0);
-        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
-            const int row = idx >> 7, f_local = idx & 127;
-            if ((row % split) != (int)rank) continue;
-            const int t = tok0 + row;
-            const long feature = (long)ft * 128 + f_local;
-            if (t >= p.M || feature >= p.N) continue;
-            float acc = 0.f;
-            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
-            if (ok) {
-                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
-                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
-            }
-        }
-        cluster_sync_all();
-    }
-    __syncthreads();
-    if (warp == 0) {
-        tc_fence_after();
-        tmem_dealloc(tmem, kTmemCols);
-    }
-}
-
-
-// --------------------------------------------------------------------------------------------------
 // TMA kernel: large token counts (prefill), channel-major X.
 // The X tile of a stage is 128 permuted channels x BN tokens.  Channel rows are fetched by the tensor
 // memory unit four arbitrary rows at a time (tile::gather4, row indices = 4 consecutive entries of the
@@ -739,16 +555,30 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
 
 
 // --------------------------------------------------------------------------------------------------
-// Streaming kernel: large token counts (prefill), channel-major X.  Same tiles and operand layouts as the
-// row-gather kernel above, but the 128 permuted channel rows of a stage are fetched by four producer
-// warps with 16-byte asynchronous copies (cp.async), 8 lanes per 128-byte row segment, which complete on
-// the stage's mbarrier.  (Measured on B200: the tensor memory unit retires one four-row gather per ~60
-// clocks, 8.5 B/clk per SM, far below what the MMA consumes; plain asynchronous row copies are not bound
-// by that.)  The epilogue transposes the accumulator tile through shared memory so that Y is written in
-// full 16-byte pieces along the feature dimension.
+// Streaming kernel: every token count, channel-major X.  A stage holds one compressed weight tile
+// (18 KB, one bulk asynchronous copy) and the matching X tile: 128 permuted channel rows x BN tokens,
+// fetched by four producer warps with 16-byte asynchronous copies (cp.async) that complete on the stage's
+// mbarrier, landing swizzled as an MN-major B operand.  (Measured on B200: the tensor memory unit retires one
+// four-row gather per ~60 clocks, 8.5 B/clk per SM, far below what the MMA consumes; plain asynchronous row
+// copies are not bound by that.)
+//
+// Decode shapes (BN = 16 / 32 / 64) are bound by the HBM stream of weight tiles, so everything is arranged
+// to get those copies in flight at once: the first weight tiles are issued by thread 0 right after it has
+// initialised the barriers, before tensor memory is allocated and before the CTA's first barrier; the grid is
+// sized so that all CTAs are resident together (no second wave); and with `static_weights` the kernel is
+// launched as a programmatic dependent of the preceding kernel on the stream, so this prologue -- which
+// touches only the weights and the permutation -- overlaps the predecessor's tail, and only the X rows
+// wait for it (griddepcontrol.wait).
+//
+// K is split across the CTAs of a cluster.  Partial tiles are reduced by pushing: token t of the tile is
+// owned by cluster rank t % split; every CTA stores its fp32 partial rows straight into the owner's
+// shared memory (slot = sender's rank) and arrives on the owner's mbarrier; the owner adds the slots in
+// rank order -- deterministic, no global scratch, one cluster-wide rendezvous at start-up only.  (Token tiles
+// of 128 and 256, whose partial tiles would not fit beside the stages, stage them in the stage area after the
+// main loop and let each owner pull its rows from the peers instead.)
 // grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192:
-//   warp 0 lane 0  weight-tile producer (bulk async copy)     warp 1 lane 0  tcgen05.cp + sparse MMAs
-//   warps 2..5     X row producers, then epilogue
+//   warp 0 lane 0  weight-tile producer        warp 1  tensor-memory allocation; lane 0: tcgen05.cp + sparse MMAs
+//   warps 2..5     X row producers, then epilogue (one quarter of the accumulator lanes each)
 // --------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -756,58 +586,198 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint3
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    return remote;
+}
+__device__ __forceinline__ void st_remote_f32(uint32_t remote_addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// Bounded wait with cluster-scope acquire (the arrivals come from other CTAs of the cluster).
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (i > 128) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
+    return false;
+}
+
+constexpr int kMaxStages = 12;
+constexpr int kPermRing = 16;        // stages of permutation entries kept ahead in shared memory
+
+// Asynchronous remote stores: the data lands in the target CTA's shared memory and its byte count completes on the
+// target's mbarrier, so the receiver needs no fence and the sender no separate arrive.
+__device__ __forceinline__ void st_async_b32(uint32_t remote_addr, uint32_t v, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote_addr), "r"(v),
+                 "r"(remote_bar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_v2(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(remote_addr),
+                 "r"(a), "r"(b), "r"(remote_bar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_v4(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                            uint32_t remote_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(remote_addr),
+                 "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar)
+                 : "memory");
+}
+__device__ __forceinline__ float4 ld_dsmem_v4(uint32_t local_addr, uint32_t rank) {
+    float4 v;
+    const uint32_t remote = map_to_rank(local_addr, rank);
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    return v;
+}
 
 template <int BN>
-__global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams p) {
-    using L = TmaCfg<BN>;
-    constexpr int STAGES = L::kStages;
+struct StreamCfg {
+    static constexpr int kRowBytes = BN >= 64 ? 128 : BN * 2;        // one channel row inside a block of <= 64 tokens
+    static constexpr int kTokBlocks = BN >= 64 ? BN / 64 : 1;
+    static constexpr int kChunks = kRowBytes / 16;                   // 16-byte pieces per row and block
+    static constexpr int kBlockBytes = 128 * kRowBytes;              // 128 channel rows of one token block
+    static constexpr int kXStage = 128 * BN * 2;
+    static constexpr int kStage = kTileBytes + kXStage;              // a multiple of 1024
+    static constexpr uint32_t kLayout = BN >= 64 ? 2u : BN == 32 ? 4u : 6u;   // 128 / 64 / 32-byte swizzle
+    static constexpr int kSwzShift = BN >= 64 ? 0 : BN == 32 ? 1 : 2;         // row bits that feed the XOR
+    static constexpr bool kPush = BN <= 64;                          // K-slice reduction by pushing (else by pulling)
+    static constexpr int kRecvBytes = kPush ? (BN + 8) * 512 : 0;    // pushed partials: [sender][128 features][rows per owner] fp32
+};
+inline size_t stream_recv_bytes(int bn, int split) { return (split > 1 && bn <= 64) ? (size_t)(bn + 8) * 512 : 0; }
+inline size_t stream_smem_bytes(int bn, int stages, int split) {
+    return (size_t)stages * (kTileBytes + 256 * bn) + stream_recv_bytes(bn, split) + kPermRing * 512 + 512 + 1024;
+}
+
+// Sends the 16 accumulator columns c0 .. c0+15 of this thread's feature to their owners (row % SPLIT), SPLIT a
+// power of two: the rows one owner gets from these 16 are consecutive in its slot, so they go as one vector.
+template <int SPLIT>
+__device__ __forceinline__ void push_columns_pow2(const uint32_t (&v)[16], int c0, uint32_t slot_local, int cnt,
+                                                  uint32_t recv_bar) {
+    constexpr int PER = 16 / SPLIT;                                  // rows per owner among 16 columns
+#pragma unroll
+    for (int o = 0; o < SPLIT; ++o) {
+        const uint32_t dst = map_to_rank(slot_local + (uint32_t)(c0 / SPLIT) * 4u, (uint32_t)o);
+        const uint32_t bar = map_to_rank(recv_bar, (uint32_t)o);
+        (void)cnt;
+        if (PER == 2) {
+            st_async_v2(dst, v[o], v[o + SPLIT], bar);
+        } else if (PER == 4) {
+            st_async_v4(dst, v[o], v[o + SPLIT], v[o + 2 * SPLIT], v[o + 3 * SPLIT], bar);
+        } else {   // PER == 8
+            st_async_v4(dst, v[o], v[o + SPLIT], v[o + 2 * SPLIT], v[o + 3 * SPLIT], bar);
+            st_async_v4(dst + 16, v[o + 4 * SPLIT], v[o + 5 * SPLIT], v[o + 6 * SPLIT], v[o + 7 * SPLIT], bar);
+        }
+    }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, const int stages) {
+    using L = StreamCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_base = sbase + L::kBarOff;
+    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
+    // layout (matches stream_smem_bytes): stages | pushed partials | permutation ring | barriers
+    const uint32_t recv_off = (uint32_t)stages * L::kStage;
+    const uint32_t perm_off = recv_off + (split > 1 ? (uint32_t)L::kRecvBytes : 0u);
+    const uint32_t bar_off = perm_off + kPermRing * 512;
+    const uint32_t bar_base = sbase + bar_off;
     auto full = [&](int s) { return bar_base + 8u * s; };
-    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
-    const uint32_t accum_bar = bar_base + 8u * 16;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 17);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 17 + 4);
+    auto empty = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+    const uint32_t accum_bar = bar_base + 8u * (2 * kMaxStages);
+    const uint32_t recv_bar = bar_base + 8u * (2 * kMaxStages + 1);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + bar_off + 8 * (2 * kMaxStages + 2));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + bar_off + 8 * (2 * kMaxStages + 2) + 4);
+    int *perm_s = reinterpret_cast<int *>(smem + perm_off);          // [kPermRing][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
-    const int split = (int)gridDim.z, slice = (int)blockIdx.z;
     const int kt_begin = slice * p.k_tiles_per_split;
     const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
     const int nk = max(0, kt_end - kt_begin);
     constexpr uint32_t kTmemCols = tmem_cols_for(BN);
+    const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
+    const int prefetch = min(stages, nk);
+    const uint32_t rank = (split > 1) ? cluster_ctarank() : 0u;
+    const int cnt = (BN + split - 1) / split;                        // rows per owner (pitch of a feature's run in a slot)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 128 + 1); mbar_init(empty(s), 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(full(s), 128 + 1); mbar_init(empty(s), 1); }
         mbar_init(accum_bar, 1);
+        mbar_init(recv_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
+        // the weight stream starts now: nothing below is needed for these copies
+        for (int it = 0; it < prefetch; ++it) {
+            mbar_arrive_expect_tx(full(it), kTileBytes);
+            bulk_load(sbase + it * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(it));
+        }
+        if (L::kPush && split > 1) {
+            // every sender delivers 128 features x (rows of this tile that this CTA owns) floats
+            const int owned = (BN - (int)rank + split - 1) / split;
+            mbar_arrive_expect_tx(recv_bar, (uint32_t)(split * owned * 512));
+        }
     }
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    if (warp >= 2) {
+        // permutation entries of the first stages, all loads in flight together (the X addresses depend on them)
+        const int g = threadIdx.x - 64;
+        int pre[kPermRing];
+#pragma unroll
+        for (int it = 0; it < kPermRing; ++it) {
+            const int kpos = (kt_begin + it) * kTileK + g;
+            pre[it] = (it < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+        }
+#pragma unroll
+        for (int it = 0; it < kPermRing; ++it) perm_s[it * 128 + g] = pre[it];
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (split > 1) cluster_arrive();       // every CTA of the cluster is running and has its barriers set up
+    grid_launch_dependents();
 
     if (warp == 0) {
         if (lane == 0) {
-            const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
-            for (int it = 0; it < nk; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+            for (int it = prefetch; it < nk; ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
                 if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
                 mbar_arrive_expect_tx(full(s), kTileBytes);
                 bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
             }
         }
+        __syncwarp();
+        if (split > 1) cluster_wait();
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
             for (int it = 0; it < nk; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
                 if (!mbar_wait(full(s), ph, abort_flag)) break;
                 fence_async_smem();          // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
                 tc_fence_after();
@@ -819,40 +789,60 @@ __global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams 
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t col = e_col + j;
                     const uint64_t ad = smem_desc(wa + j * 32, 16, 1024, kLayoutSw128);
-                    const uint64_t bd = smem_desc(xa + j * 4096, 16384, 1024, kLayoutSw128);
+                    const uint64_t bd = (BN >= 64) ? smem_desc(xa + j * 4096, L::kBlockBytes, 1024, kLayoutSw128)
+                                                   : smem_desc(xa + j * 32 * L::kRowBytes, 8 * L::kRowBytes, 8 * L::kRowBytes, L::kLayout);
                     tc_mma_sparse_f16(tmem, ad, bd, tmem + (col & ~1u), idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
                 }
                 tc_commit(empty(s));
             }
             tc_commit(accum_bar);
         }
+        __syncwarp();
+        if (split > 1) cluster_wait();
     } else {
-        // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) + 16 i of every 64-token block
+        // ---- X producers: thread g copies the 16-byte pieces e = g, g + 128, ... of the stage's 128 rows
         const int g = threadIdx.x - 64;
-        const int cc = g & 7, rg = g >> 3;
+        constexpr int kPieces = 128 * L::kChunks;                     // per token block
+        constexpr int kPerThread = (kPieces + 127) / 128;
         const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
+        const bool ring_refill = nk > kPermRing;                      // long K-slices: keep the ring kPermRing stages ahead
         bool alive = true;
+        int refill = -1;
+        grid_dependency_wait();                                       // X may come from the preceding kernel
         for (int it = 0; it < nk; ++it) {
-            const int s = it % STAGES;
-            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-            int ch[8];
+            const int s = it % stages;
+            const uint32_t ph = (uint32_t)(it / stages) & 1u;
+            const int *pr = perm_s + (it % kPermRing) * 128;
+            if (ring_refill && it > 0) perm_s[((it - 1) % kPermRing) * 128 + g] = refill;   // entries of stage it-1+kPermRing
+            int ch[kPerThread];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int kpos = (kt_begin + it) * kTileK + rg + 16 * i;
-                ch[i] = (kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+            for (int i = 0; i < kPerThread; ++i) {
+                const int e = g + 128 * i;
+                ch[i] = (e < kPieces) ? pr[e / L::kChunks] : -1;
             }
-            if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+            if (ring_refill) {
+                asm volatile("bar.sync 1, 128;" ::: "memory");       // everyone has read this stage's entries
+                const int kpos = (kt_begin + it + kPermRing) * kTileK + g;
+                refill = (it + kPermRing < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+            }
+            // (a thread whose wait gave up keeps looping without copying: the named barrier above needs all 128)
+            if (alive && !mbar_wait(empty(s), ph ^ 1u, abort_flag)) alive = false;
+            if (!alive) continue;
             const uint32_t xs = sbase + s * L::kStage + kTileBytes;
 #pragma unroll
-            for (int tb = 0; tb < BN / 64; ++tb) {
-                const int t = tok0 + tb * 64 + cc * 8;
-                const int valid = min(8, max(0, p.M - t));
+            for (int tb = 0; tb < L::kTokBlocks; ++tb) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = rg + 16 * i;
-                    const bool in = ch[i] >= 0 && valid > 0;
-                    const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
-                    cp_async_16(xs + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4), src, in ? valid * 2 : 0);
+                for (int i = 0; i < kPerThread; ++i) {
+                    const int e = g + 128 * i;
+                    if (e < kPieces) {
+                        const int r = e / L::kChunks, cc = e % L::kChunks;
+                        const int t = tok0 + tb * 64 + cc * 8;
+                        const int valid = min(8, max(0, p.M - t));
+                        const bool in = ch[i] >= 0 && valid > 0;
+                        const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
+                        const int cs = cc ^ ((r >> L::kSwzShift) & (L::kChunks - 1));
+                        cp_async_16(xs + tb * L::kBlockBytes + r * L::kRowBytes + (cs << 4), src, in ? valid * 2 : 0);
+                    }
                 }
             }
             cp_async_arrive_noinc(full(s));
@@ -860,7 +850,7 @@ __global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams 
         // ---- epilogue
         const int quarter = warp & 3;
         const int f_local = quarter * 32 + lane;
-        const bool ok = alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
+        const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
         tc_fence_after();
         if (split == 1) {
             // accumulators -> shared memory [token][128 features] in the output type -> 16-byte stores
@@ -868,7 +858,7 @@ __global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams 
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 uint32_t v[16];
-                if (nk > 0) {
+                if (nk > 0 && ok) {
                     tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
                 } else {
 #pragma unroll
@@ -906,12 +896,14 @@ __global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams 
                         }
                 }
             }
-        } else {
+        } else if (!L::kPush) {
+            // ---- stage the fp32 partial tile [token][128 features]; owners pull after the cluster barrier below
+            cluster_wait();
             float *stage_f32 = reinterpret_cast<float *>(smem);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 uint32_t v[16];
-                if (nk > 0) {
+                if (nk > 0 && ok) {
                     tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
                 } else {
 #pragma unroll
@@ -921,45 +913,119 @@ __global__ void __launch_bounds__(192, 1) spgemm_stream_kernel(const GemmParams 
                 for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
             }
             tc_fence_before();
-        }
-    }
-
-    if (split > 1) {
-        cluster_sync_all();
-        const uint32_t rank = cluster_ctarank();
-        const bool ok = (*abort_flag == 0);
-        for (int idx = threadIdx.x; idx < BN * 128; idx += 192) {
-            const int row = idx >> 7, f_local = idx & 127;
-            if ((row % split) != (int)rank) continue;
-            const int t = tok0 + row;
-            const long feature = (long)ft * 128 + f_local;
-            if (t >= p.M || feature >= p.N) continue;
-            float acc = 0.f;
-            for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
-            if (ok) {
-                if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
-                else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
+        } else {
+            // ---- push the partial rows to their owners (row % split), then finish the rows this CTA owns
+            cluster_wait();                                          // all CTAs of the cluster have initialised their barriers
+            const uint32_t slot_local = sbase + recv_off + (uint32_t)(((int)rank * 128 + f_local) * cnt) * 4u;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t v[16];
+                if (nk > 0 && ok) {
+                    tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0;
+                }
+                if (split == 2) push_columns_pow2<2>(v, c0, slot_local, cnt, recv_bar);
+                else if (split == 4) push_columns_pow2<4>(v, c0, slot_local, cnt, recv_bar);
+                else if (split == 8) push_columns_pow2<8>(v, c0, slot_local, cnt, recv_bar);
+                else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int row = c0 + e;
+                        const uint32_t owner = (uint32_t)(row % split);
+                        st_async_b32(map_to_rank(slot_local + (uint32_t)(row / split) * 4u, owner), v[e],
+                                     map_to_rank(recv_bar, owner));
+                    }
+                }
+            }
+            tc_fence_before();
+            const bool got = mbar_wait_cluster(recv_bar, 0, abort_flag);
+            const bool fine = got && (*abort_flag == 0);
+            const float *recv = reinterpret_cast<const float *>(smem + recv_off);
+            const int f_valid = min(128, p.N - ft * 128);
+            const int owned = (BN - (int)rank + split - 1) / split;
+            for (int q = g; q < owned * 128; q += 128) {
+                const int i = q >> 7, f = q & 127;
+                const int t = tok0 + i * split + (int)rank;
+                if (!fine || t >= p.M || f >= f_valid) continue;
+                float acc = 0.f;
+                for (int r = 0; r < split; ++r) acc += recv[(r * 128 + f) * cnt + i];   // slice order: deterministic
+                const long o = (long)t * p.ldy + (long)ft * 128 + f;
+                if (p.out_f32) reinterpret_cast<float *>(p.Y)[o] = acc;
+                else reinterpret_cast<__half *>(p.Y)[o] = __float2half_rn(acc);
             }
         }
-        cluster_sync_all();
+    }
+    if (!L::kPush && split > 1) {
+        cluster_sync_all();                                          // every partial tile is staged
+        const bool fine = (*abort_flag == 0);
+        const int f_valid = min(128, p.N - ft * 128);
+        for (int q = threadIdx.x; q < BN * 32; q += 192) {            // 4 consecutive features of one row per thread
+            const int row = q >> 5, f0 = (q & 31) * 4;
+            if ((row % split) != (int)rank) continue;
+            const int t = tok0 + row;
+            if (t >= p.M || f0 >= f_valid) continue;
+            float4 part[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+                if (r < split) part[r] = ld_dsmem_v4(sbase + (uint32_t)(row * 128 + f0) * 4u, (uint32_t)r);
+            float a[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+                if (r < split) { a[0] += part[r].x; a[1] += part[r].y; a[2] += part[r].z; a[3] += part[r].w; }   // slice order
+            if (fine) {
+                const long o = (long)t * p.ldy + (long)ft * 128 + f0;
+                for (int e = 0; e < 4; ++e)
+                    if (f0 + e < f_valid) {
+                        if (p.out_f32) reinterpret_cast<float *>(p.Y)[o + e] = a[e];
+                        else reinterpret_cast<__half *>(p.Y)[o + e] = __float2half_rn(a[e]);
+                    }
+            }
+        }
+        cluster_sync_all();                                          // nobody leaves while a peer still reads its tile
     }
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
 }
 
 template <int BN>
-esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int split, cudaStream_t stream) {
-    using L = TmaCfg<BN>;
+esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int split, int stages, bool dependent,
+                           cudaStream_t stream) {
     auto kern = spgemm_stream_kernel<BN>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    const size_t smem = stream_smem_bytes(BN, stages, split);
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(f_tiles, t_tiles, split);
     cfg.blockDim = dim3(192);
-    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, stages));
+    return ESP_OK;
+}
+
+// Clusters of `split` CTAs of the streaming kernel that can be resident at once on this device.
+template <int BN>
+int stream_cluster_capacity(int split, int stages) {
+    auto kern = spgemm_stream_kernel<BN>;
+    const size_t smem = stream_smem_bytes(BN, stages, split);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, 1, split);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
@@ -967,8 +1033,9 @@ esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int sp
     attr[0].val.clusterDim.z = split;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
-    return ESP_OK;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -1020,31 +1087,6 @@ esp_status_t launch_tma(const GemmParams &p, int f_tiles, int t_tiles, int split
     return ESP_OK;
 }
 
-inline size_t resident_smem_bytes(int bn, int stages, int k_tiles_per_split) {
-    return (size_t)stages * kTileBytes + (size_t)k_tiles_per_split * 128 * bn * 2 + 256 + 1024;
-}
-
-template <int BN>
-esp_status_t launch_resident(const GemmParams &p, int f_tiles, int t_tiles, int split, int stages, cudaStream_t stream) {
-    auto kern = spgemm_resident_kernel<BN>;
-    const size_t smem = resident_smem_bytes(BN, stages, p.k_tiles_per_split);
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(f_tiles, t_tiles, split);
-    cfg.blockDim = dim3(192);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = split;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, stages));
-    return ESP_OK;
-}
-
 // [M, K] token-major -> [K, ldt] channel-major (a transposed, not permuted, copy; ldt >= M).
 __global__ void __launch_bounds__(256) transpose_x_kernel(const uint16_t *__restrict__ X, int M, int K, long ldx,
                                                           uint16_t *__restrict__ Xt, long ldt) {
@@ -1073,6 +1115,29 @@ size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
     return align_up((size_t)K * (size_t)transposed_ld(M) * 2, 256);
 }
 
+// Resident capacity (in CTAs) of the streaming kernel for one configuration, cached per process.
+static int stream_capacity_ctas(int bn, int split, int stages) {
+    static std::mutex mu;
+    static std::map<long, int> cache;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const long key = (((long)dev * 512 + bn) * 16 + split) * 16 + stages;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int clusters = 0;
+    switch (bn) {
+        case 16: clusters = stream_cluster_capacity<16>(split, stages); break;
+        case 32: clusters = stream_cluster_capacity<32>(split, stages); break;
+        case 64: clusters = stream_cluster_capacity<64>(split, stages); break;
+        case 128: clusters = stream_cluster_capacity<128>(split, stages); break;
+        case 256: clusters = stream_cluster_capacity<256>(split, stages); break;
+        default: break;
+    }
+    cache[key] = clusters * split;
+    return clusters * split;
+}
+
 esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan) {
     DeviceInfo di;
     esp_status_t st = device_info(&di);
@@ -1083,51 +1148,63 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
     const bool channel_major_available = (o.x_layout == ESP_X_CHANNEL_MAJOR) || have_workspace;
     int bn = o.token_tile;
     g.kernel = ESP_KERNEL_GATHER;
-    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available) {
-        const bool small = M <= 64 && (bn == 0 || bn <= 64);
-        if (o.force_kernel == ESP_KERNEL_RESIDENT) g.kernel = small ? ESP_KERNEL_RESIDENT : ESP_KERNEL_GATHER;
-        else if (o.force_kernel == ESP_KERNEL_TMA) g.kernel = ESP_KERNEL_TMA;
-        else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
-        else g.kernel = small ? ESP_KERNEL_RESIDENT : ESP_KERNEL_STREAM;
-    }
-    const bool tiled = (g.kernel == ESP_KERNEL_TMA || g.kernel == ESP_KERNEL_STREAM);
-    if (tiled && bn != 0 && bn < 64) bn = 64;
+    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available)
+        g.kernel = (o.force_kernel == ESP_KERNEL_TMA) ? ESP_KERNEL_TMA : ESP_KERNEL_STREAM;
     if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-    if (tiled && bn < 64) bn = 64;
+    if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
-    const int t_tiles = ceil_div(M, bn);
-    int split = o.split_k;
     g.stages = 4;
-    if (g.kernel == ESP_KERNEL_RESIDENT) {
-        // the K-slice of X must fit beside the weight stages; more slices also spread the weight stream
-        const size_t x_cap = 64 * 1024;
-        int min_split = 1;
-        while (min_split < 8 && (size_t)ceil_div(k_tiles, min_split) * 128 * bn * 2 > x_cap) ++min_split;
-        if (split == 0) {
-            split = min_split;
-            while (split < 8 && (long)f_tiles * t_tiles * split < 2L * di.sm_count && ceil_div(k_tiles, split + 1) >= 2) ++split;
+    const int t_tiles = ceil_div(M, bn);
+    const long tiles = (long)f_tiles * t_tiles;
+    auto no_empty_slice = [&](int split) { return (long)ceil_div(k_tiles, split) * (split - 1) < k_tiles; };
+    if (g.kernel == ESP_KERNEL_STREAM) {
+        // Pick K-slices and CTAs per SM so that, if possible, the whole grid is resident at once and each CTA
+        // has a short chain of tiles: cost ~ waves x (tiles per CTA + fixed start-up and reduction time).
+        const size_t per_stage = (size_t)kTileBytes + 256 * (size_t)bn;
+        double best_cost = 1e30;
+        int best_split = 0, best_stages = 0;
+        int wanted = o.split_k > k_tiles ? k_tiles : o.split_k;      // a requested split steps down to one without empty slices
+        while (wanted > 1 && !no_empty_slice(wanted)) --wanted;
+        for (int split = 1; split <= 8 && split <= k_tiles; ++split) {
+            if (wanted != 0 && split != wanted) continue;
+            if (!no_empty_slice(split)) continue;
+            const int kts = ceil_div(k_tiles, split);
+            const size_t fixed = stream_recv_bytes(bn, split) + kPermRing * 512 + 512 + 1024;
+            int last_stages = -1;
+            for (int r = 1; r <= 4; ++r) {
+                const size_t budget = (size_t)di.max_smem_optin / r - (r > 1 ? 1024 : 0);
+                if (budget < fixed + 2 * per_stage) break;
+                int stages = (int)((budget - fixed) / per_stage);
+                if (stages > kMaxStages) stages = kMaxStages;
+                if (stages > kts) stages = kts < 2 ? 2 : kts;
+                if (stages == last_stages) continue;
+                last_stages = stages;
+                const int cap = stream_capacity_ctas(bn, split, stages);
+                if (cap <= 0) continue;
+                const long ctas = tiles * split;
+                const long waves = (ctas + cap - 1) / cap;
+                double cost = (double)waves * (kts + 2.0) + (split > 1 ? 0.25 + 0.05 * split : 0.0) + 0.01 * r;
+                // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
+                if (o.static_weights && 2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin) cost += 3.0;
+                if (cost < best_cost) { best_cost = cost; best_split = split; best_stages = stages; }
+            }
         }
-        if (split < min_split) split = min_split;
-        if ((size_t)ceil_div(k_tiles, split) * 128 * bn * 2 > 96 * 1024) g.kernel = ESP_KERNEL_GATHER;
+        if (best_split == 0) return ESP_ERR_UNSUPPORTED;
+        g.split_k = best_split;
+        g.stages = best_stages;
+        *plan = g;
+        return ESP_OK;
     }
-    if (g.kernel != ESP_KERNEL_RESIDENT && split == 0) {
+    int split = o.split_k;
+    if (split == 0) {
         split = 1;
-        while (split < 8 && (long)f_tiles * t_tiles * split < di.sm_count && k_tiles / (split * 2) >= 4) split *= 2;
+        while (split < 8 && tiles * split < di.sm_count && k_tiles / (split * 2) >= 4) split *= 2;
     }
     if (split > k_tiles) split = k_tiles;
     if (split < 1) split = 1;
-    while (split > 1 && (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles) --split;   // no empty slice
+    while (split > 1 && !no_empty_slice(split)) --split;
     g.split_k = split;
-    if (g.kernel == ESP_KERNEL_RESIDENT) {
-        const size_t xbytes = (size_t)ceil_div(k_tiles, split) * 128 * bn * 2;
-        const long ctas = (long)f_tiles * t_tiles * split;
-        const size_t budget = (ctas > di.sm_count ? 112 : 220) * 1024 - 2048;
-        int stages = (int)((budget - (xbytes < budget ? xbytes : budget)) / kTileBytes);
-        if (stages > 8) stages = 8;
-        if (stages < 2) stages = 2;
-        g.stages = stages;
-    }
     *plan = g;
     return ESP_OK;
 }
@@ -1157,26 +1234,21 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.ldx = ldt;
             p.x_channel_major = 1;
         }
+        const bool dependent = o.static_weights != 0;
         if (plan.kernel == ESP_KERNEL_STREAM) {
             switch (plan.token_tile) {
-                case 64: return launch_stream<64>(p, f_tiles, t_tiles, plan.split_k, stream);
-                case 128: return launch_stream<128>(p, f_tiles, t_tiles, plan.split_k, stream);
-                case 256: return launch_stream<256>(p, f_tiles, t_tiles, plan.split_k, stream);
-                default: return ESP_ERR_INVALID_ARG;
-            }
-        }
-        if (plan.kernel == ESP_KERNEL_TMA) {
-            switch (plan.token_tile) {
-                case 64: return launch_tma<64>(p, f_tiles, t_tiles, plan.split_k, stream);
-                case 128: return launch_tma<128>(p, f_tiles, t_tiles, plan.split_k, stream);
-                case 256: return launch_tma<256>(p, f_tiles, t_tiles, plan.split_k, stream);
+                case 16: return launch_stream<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);
+                case 32: return launch_stream<32>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);
+                case 64: return launch_stream<64>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);
+                case 128: return launch_stream<128>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);
+                case 256: return launch_stream<256>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);
                 default: return ESP_ERR_INVALID_ARG;
             }
         }
         switch (plan.token_tile) {
-            case 16: return launch_resident<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
-            case 32: return launch_resident<32>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
-            case 64: return launch_resident<64>(p, f_tiles, t_tiles, plan.split_k, plan.stages, stream);
+            case 64: return launch_tma<64>(p, f_tiles, t_tiles, plan.split_k, stream);
+            case 128: return launch_tma<128>(p, f_tiles, t_tiles, plan.split_k, stream);
+            case 256: return launch_tma<256>(p, f_tiles, t_tiles, plan.split_k, stream);
             default: return ESP_ERR_INVALID_ARG;
         }
     }

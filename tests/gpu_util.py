@@ -56,7 +56,7 @@ def pack_on_gpu(vals, meta):
 
 
 def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0, token_tile=0, kernel=0,
-           workspace=True):
+           workspace=True, static_weights=0):
     dev = torch.device(DEV)
     M = X.shape[0]
     Xd = torch.from_numpy(np.ascontiguousarray(X)).to(dev)
@@ -70,6 +70,7 @@ def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0
     o.x_layout = b.ESP_X_CHANNEL_MAJOR if channel_major else b.ESP_X_TOKEN_MAJOR
     o.out_dtype = b.ESP_OUT_F32 if out_f32 else b.ESP_OUT_F16
     o.split_k, o.token_tile, o.force_kernel = split_k, token_tile, kernel
+    o.static_weights = static_weights
     Y = torch.full((M, N), float("nan"), dtype=torch.float32 if out_f32 else torch.float16, device=dev)
     th = None if theta is None else torch.from_numpy(np.ascontiguousarray(theta, dtype=np.int32)).to(dev)
     ws = None

@@ -53,7 +53,8 @@ def test_config0_all_variants():
     for kw in (dict(), dict(split_k=2), dict(split_k=4, out_f32=True), dict(channel_major=True),
                dict(token_tile=64), dict(token_tile=16, split_k=4), dict(token_tile=256, out_f32=True),
                dict(token_tile=64, channel_major=True, split_k=2), dict(token_tile=32, workspace=True),
-               dict(kernel=1, workspace=False), dict(kernel=1, channel_major=True, token_tile=128)):
+               dict(kernel=1, workspace=False), dict(kernel=1, channel_major=True, token_tile=128),
+               dict(static_weights=1), dict(static_weights=1, channel_major=True, split_k=4, token_tile=32)):
         check(spgemm(X, packed, ref.theta, 512, **kw), Yref, kw.get("out_f32", False))
 
 
@@ -70,6 +71,7 @@ def test_decode_and_ragged_shapes(M, N, K):
     check(spgemm(X, packed, theta, N, split_k=3, out_f32=True), Yref, True)
     check(spgemm(X, packed, theta, N, channel_major=True), Yref)
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=1, split_k=2), Yref)
+    check(spgemm(X, packed, theta, N, channel_major=True, static_weights=1, split_k=5), Yref)
 
 
 @pytest.mark.parametrize("kernel", [4, 2])
@@ -114,6 +116,34 @@ def test_split_k_is_deterministic_and_order_fixed():
     for _ in range(3):
         assert np.array_equal(a, spgemm(X, packed, theta, 256, split_k=8, out_f32=True))
     check(a, orc.product(X, vals, meta, theta), True)
+
+
+def test_chain_of_dependent_launches_with_static_weights():
+    """Six layers back to back on one stream, each reading the previous layer's output, launched with
+    static_weights = 1 (weight prefetch overlapping the predecessor's tail): every layer's result must equal
+    the oracle's product of that layer's actual input, i.e. no layer may read its input early."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    N = K = 1024
+    M = 16
+    vals, meta, theta = pruned(77, N, K)
+    vals = (vals.astype(np.float32) * 1.7).astype(np.float16)      # keeps the activations O(1) through the chain
+    packed = pack_on_gpu(vals, meta)
+    dev = torch.device("cuda:0")
+    th = torch.from_numpy(theta).to(dev)
+    X0 = np.random.default_rng(3).standard_normal((M, K)).astype(np.float16)
+    acts = [torch.from_numpy(X0).to(dev)] + [torch.empty(M, N, dtype=torch.float16, device=dev) for _ in range(6)]
+    o = b.esp_gemm_opts_default()
+    o.static_weights = 1
+    ws = torch.empty(b.esp_spgemm_workspace_bytes(M, N, K, o), dtype=torch.uint8, device=dev)
+    for rep in range(3):
+        for i in range(6):
+            b.esp_spgemm(acts[i], packed, th, acts[i + 1], o, ws)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    for i in range(6):
+        check(acts[i + 1].cpu().numpy(), orc.product(acts[i].cpu().numpy(), vals, meta, theta))
 
 
 def test_llama7b_shapes_sampled_outputs():
