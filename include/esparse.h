@@ -141,8 +141,10 @@ enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_TMA = 2,       /* channel-major X rows fetched four at a time by the tensor memory
                                     unit's row gather (correct, but that unit retires such gathers too
                                     slowly to feed the MMA; kept for comparison)                        */
-       ESP_KERNEL_STREAM = 4 };  /* channel-major X rows streamed by asynchronous 16-byte copies, weight
-                                    tiles by bulk copies; every token count (the default)               */
+       ESP_KERNEL_STREAM = 4,    /* channel-major X rows streamed by asynchronous 16-byte copies, weight
+                                    tiles by bulk copies; every token count (default up to 256 tokens)  */
+       ESP_KERNEL_PAIR = 5 };    /* large M: two SMs share one 512-feature x token_tile MMA tile
+                                    (token_tile 240 by default; 128, 192, 224 or 256 on request)        */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
@@ -150,7 +152,8 @@ typedef struct {
     int out_dtype;               /* ESP_OUT_*: type of Y                                              */
     int split_k;                 /* K-slices reduced inside a thread-block cluster; 0 = choose, 1..8  */
     int force_kernel;            /* ESP_KERNEL_*                                                      */
-    int token_tile;              /* tokens per CTA tile (16, 32, 64, 128 or 256); 0 = choose          */
+    int token_tile;              /* tokens per tile (16, 32, 64, 128 or 256; pair kernel: see above);
+                                    0 = choose                                                        */
     int static_weights;          /* 1 = `packed` and `perm` are not written by work still pending on the
                                     stream (the usual case at inference).  The kernel is then launched as
                                     a programmatic dependent of the preceding kernel: its weight prefetch

@@ -18,7 +18,7 @@ ESP_ERR_STATIC_LIMIT = 8
 ESP_STATIC_SCRATCH_BYTES = 8 << 20
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
-ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM = 0, 1, 2, 4
+ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR = 0, 1, 2, 4, 5
 
 
 class esp_prune_opts(ctypes.Structure):

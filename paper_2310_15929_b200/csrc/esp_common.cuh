@@ -66,7 +66,7 @@ esp_status_t launch_decompress(const __half *vals, const uint8_t *meta, const in
 
 // ---- GEMM launchers (spgemm_kernels.cu) ------------------------------------------------------------
 struct GemmPlan {
-    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA | ESP_KERNEL_STREAM
+    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA | ESP_KERNEL_STREAM | ESP_KERNEL_PAIR
     int token_tile;    // MMA N
     int split_k;       // cluster size along K
     int stages;

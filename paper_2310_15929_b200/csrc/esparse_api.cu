@@ -42,7 +42,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
     if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
-        o->force_kernel != ESP_KERNEL_STREAM)
+        o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;

@@ -1038,6 +1038,8 @@ int stream_cluster_capacity(int split, int stages) {
     return n;
 }
 
+#include "spgemm_pair.cuh"
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1148,8 +1150,21 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
     const bool channel_major_available = (o.x_layout == ESP_X_CHANNEL_MAJOR) || have_workspace;
     int bn = o.token_tile;
     g.kernel = ESP_KERNEL_GATHER;
-    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available)
-        g.kernel = (o.force_kernel == ESP_KERNEL_TMA) ? ESP_KERNEL_TMA : ESP_KERNEL_STREAM;
+    if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available) {
+        if (o.force_kernel == ESP_KERNEL_TMA) g.kernel = ESP_KERNEL_TMA;
+        else if (o.force_kernel == ESP_KERNEL_PAIR) g.kernel = ESP_KERNEL_PAIR;
+        else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
+        else g.kernel = (M > 256 && o.split_k <= 1) ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;   // the pair kernel has no K-slices
+    }
+    if (g.kernel == ESP_KERNEL_PAIR) {
+        if (bn == 0) bn = 240;
+        if (bn != 128 && bn != 192 && bn != 224 && bn != 240 && bn != 256) return ESP_ERR_INVALID_ARG;
+        g.token_tile = bn;
+        g.split_k = 1;
+        g.stages = 0;
+        *plan = g;
+        return ESP_OK;
+    }
     if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
     if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
@@ -1235,6 +1250,16 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.x_channel_major = 1;
         }
         const bool dependent = o.static_weights != 0;
+        if (plan.kernel == ESP_KERNEL_PAIR) {
+            switch (plan.token_tile) {
+                case 128: return launch_pair<2, 128>(p, stream);
+                case 192: return launch_pair<2, 192>(p, stream);
+                case 224: return launch_pair<2, 224>(p, stream);
+                case 240: return launch_pair<2, 240>(p, stream);
+                case 256: return launch_pair<1, 256>(p, stream);
+                default: return ESP_ERR_INVALID_ARG;
+            }
+        }
         if (plan.kernel == ESP_KERNEL_STREAM) {
             switch (plan.token_tile) {
                 case 16: return launch_stream<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, dependent, stream);

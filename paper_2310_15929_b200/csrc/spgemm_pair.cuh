@@ -1,0 +1,333 @@
+// Pair kernel: large token counts (prefill), channel-major X.  Included by spgemm_kernels.cu inside
+// namespace esp { namespace { ... } } after the helpers it uses.
+//
+// At the sparse tensor-core rate a CTA consumes a 128-channel step of a 128-feature x 256-token tile in 512
+// clocks; filling shared memory for it (18 KB of weights + 64 KB of gathered X rows) would need 164 B/clk
+// per SM, several times what an SM can pull in.  So the tile is made as large as tensor memory allows and is
+// shared by two SMs:
+//
+//   * a cluster of two CTAs issues one MMA of 256 features x TN tokens (tcgen05.mma.sp.cta_group::2): each CTA
+//     supplies its own 128 feature rows of the compressed weight and HALF of the tokens of the X tile;
+//   * each CTA carries NA = 2 such accumulators (2 x TN fp32 columns of tensor memory + metadata columns use
+//     all 512), so the pair covers 512 features x TN tokens and an X row is gathered once for 512 features.
+//
+// With TN = 240 a 128-channel step moves 36 KB of weight tiles (bulk asynchronous copies) and 30 KB of X rows
+// (16-byte asynchronous copies) per CTA for 960 clocks of MMA: 70 B/clk per SM instead of 164.
+//
+// Two measured properties of the SM's copy paths shape the producers (B200, data resident in L2):
+//   * bulk copies issued by ONE thread complete one after the other, about 0.45 us each whatever their size
+//     (18 KB copies: 41 GB/s per SM from one thread, 81 from two, 134 from four), so the weight tiles of a
+//     stage are issued by different lanes;
+//   * 16-byte asynchronous row copies deliver about 25 GB/s per SM from 128 threads, 44 from 256 and 60 from
+//     512, independent of how many stages are in flight, so sixteen warps gather X.
+//
+// grid (2 x feature-pair tiles, token tiles, 1), cluster (2,1,1), block 576.  In both CTAs:
+//   warp 0 lanes 0..3  weight-tile producers (tile copies dealt round-robin)
+//   warp 1             tensor-memory allocation; lane 0 of the leader CTA (rank 0): tcgen05.cp + MMAs for the pair;
+//                      lane 0 of rank 1: forwards "my stage is full" to the leader's barrier
+//   warps 2..17        X row producers, then epilogue (four warps per quarter of the accumulator lanes)
+// A stage's `empty` barrier and the final `accum` barrier are signalled in both CTAs at once by
+// tcgen05.commit with a CTA mask.  No load uses cluster multicast.
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in every CTA of the mask once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(cta_mask)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_copy_128x128b_pair(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_sparse_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t e_tmem,
+                                                       uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+constexpr int kPairProducers = 512;                  // X producer threads (warps 2..17)
+constexpr int kPairThreads = 64 + kPairProducers;
+constexpr int kPairIssuers = 4;                      // lanes of warp 0 that issue weight-tile copies
+
+template <int NA, int TN>
+struct PairCfg {
+    static constexpr int kHalf = TN / 2;                              // tokens of X each CTA stages
+    static constexpr int kTokBlocks = (kHalf + 63) / 64;              // 64-token blocks of 128 rows x 128 bytes
+    static constexpr int kXStage = kTokBlocks * 16384;
+    static constexpr int kWStage = NA * kTileBytes;
+    static constexpr int kStage = kWStage + kXStage;                  // a multiple of 1024
+    static constexpr int kStagesFit = (227 * 1024 - kPermRing * 512 - 512 - 1024) / kStage;
+    static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
+    static constexpr int kPermOff = kStages * kStage;
+    static constexpr int kBarOff = kPermOff + kPermRing * 512;
+    static constexpr int kTotal = kBarOff + 512 + 1024;
+    static constexpr uint32_t kTmemCols = 512;
+    static_assert(NA * 256 <= 512 && TN + 8 <= 256 + (NA == 1 ? 8 : 0) && TN % 16 == 0, "tensor memory layout");
+    __host__ __device__ static constexpr uint32_t acc_col(int a) { return (uint32_t)a * 256u; }
+    __host__ __device__ static constexpr uint32_t meta_col(int a, int buf) { return (uint32_t)a * 256u + TN + 4u * buf; }
+};
+
+template <int NA, int TN>
+__global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p) {
+    using L = PairCfg<NA, TN>;
+    constexpr int STAGES = L::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + L::kBarOff;
+    auto full = [&](int s) { return bar_base + 8u * s; };
+    auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
+    auto peer_full = [&](int s) { return bar_base + 8u * (16 + s); };    // used in the leader only
+    const uint32_t accum_bar = bar_base + 8u * 24;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
+    int *perm_s = reinterpret_cast<int *>(smem + L::kPermOff);           // [kPermRing][128]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                              // 0 = leader
+    const int pair_idx = (int)blockIdx.x >> 1;
+    const int tok0 = (int)blockIdx.y * TN;                                // first token of the pair's tile
+    const int tok_cta = tok0 + (int)rank * L::kHalf;                      // first token this CTA stages
+    const int nk = p.k_tiles;
+    const int f_tiles = (p.N + 127) / 128;
+    int ftile[NA];
+    bool present[NA];
+    int n_present = 0;
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        ftile[a] = pair_idx * (2 * NA) + 2 * a + (int)rank;               // MMA a: rows 0..127 from rank 0, 128..255 from rank 1
+        present[a] = ftile[a] < f_tiles;
+        n_present += present[a] ? 1 : 0;
+    }
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full(s), kPairProducers + (uint32_t)n_present);    // X threads + one arrival per weight-tile copy
+            mbar_init(empty(s), 1);
+            mbar_init(peer_full(s), 1);
+        }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), L::kTmemCols);
+    // a feature tile beyond N: zero values and legal metadata once, never loaded
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        if (!present[a]) {
+            for (int s = 0; s < STAGES; ++s) {
+                uint32_t *dst = reinterpret_cast<uint32_t *>(smem + s * L::kStage + a * kTileBytes);
+                for (int i = threadIdx.x; i < kTileBytes / 4; i += kPairThreads) dst[i] = (i < kTileValBytes / 4) ? 0u : 0x44444444u;
+            }
+        }
+    }
+    if (warp >= 2) {
+        // permutation entries of the first kPermRing stages: thread g takes row g % 128 of stages g / 128 + 4 i
+        const int g = threadIdx.x - 64;
+        int pre[kPermRing / 4];
+#pragma unroll
+        for (int i = 0; i < kPermRing / 4; ++i) {
+            const int it = (g >> 7) + 4 * i;
+            const int kpos = it * kTileK + (g & 127);
+            pre[i] = (it < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+        }
+#pragma unroll
+        for (int i = 0; i < kPermRing / 4; ++i) perm_s[((g >> 7) + 4 * i) * 128 + (g & 127)] = pre[i];
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                      // both CTAs have their barriers and tensor memory before any cross-CTA signal
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane < kPairIssuers) {
+            // copy number q = it * NA + a goes to lane q % kPairIssuers (copies of one thread do not overlap)
+            for (int q = lane; q < nk * NA; q += kPairIssuers) {
+                const int it = q / NA, a = q % NA;
+                if (!present[a]) continue;
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(full(s), kTileBytes);
+                bulk_load(sbase + s * L::kStage + a * kTileBytes, p.packed + ((long)ftile[a] * p.k_tiles + it) * kTileBytes,
+                          kTileBytes, full(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank != 0) {
+            // forward "my operands of this stage have landed" to the leader
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(full(s), ph, abort_flag)) break;
+                fence_async_smem();          // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
+                mbar_arrive_remote(map_to_rank(peer_full(s), 0));
+            }
+        } else if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_sparse_f16(256, TN, 1);
+            for (int it = 0; it < nk; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (!mbar_wait(full(s), ph, abort_flag)) break;
+                if (!mbar_wait_cluster(peer_full(s), ph, abort_flag)) break;
+                fence_async_smem();
+                tc_fence_after();
+                const uint32_t wa = sbase + s * L::kStage;
+                const uint32_t xa = wa + L::kWStage;
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    const uint32_t e_col = L::meta_col(a, it & 1);
+                    const uint32_t ta = wa + a * kTileBytes;
+                    tc_copy_128x128b_pair(tmem + e_col, smem_desc(ta + kTileValBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t col = e_col + j;
+                        const uint64_t ad = smem_desc(ta + j * 32, 16, 1024, kLayoutSw128);
+                        const uint64_t bd = smem_desc(xa + j * 4096, 16384, 1024, kLayoutSw128);
+                        tc_mma_sparse_f16_pair(tmem + L::acc_col(a), ad, bd, tmem + (col & ~1u), idesc | (col & 1u),
+                                               (it > 0 || j > 0) ? 1u : 0u);
+                    }
+                }
+                tc_commit_pair(empty(s), (uint16_t)3);
+            }
+            tc_commit_pair(accum_bar, (uint16_t)3);
+        }
+    } else {
+        // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) and (g >> 3) + 64 of every 64-token block
+        const int g = threadIdx.x - 64;
+        const int cc = g & 7, rg = g >> 3;
+        const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
+        const bool ring_refill = nk > kPermRing;
+        bool alive = true;
+        int refill = -1;
+        for (int it = 0; it < nk; ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+            const int *pr = perm_s + (it % kPermRing) * 128;
+            if (ring_refill && it > 0 && g < 128) perm_s[((it - 1) % kPermRing) * 128 + g] = refill;   // stage it-1+kPermRing
+            int ch[2];
+            ch[0] = pr[rg];
+            ch[1] = pr[rg + 64];
+            if (ring_refill) {
+                asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");   // everyone has read this stage's entries
+                if (g < 128) {
+                    const int kpos = (it + kPermRing) * kTileK + g;
+                    refill = (it + kPermRing < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+                }
+            }
+            if (alive && !mbar_wait(empty(s), ph ^ 1u, abort_flag)) alive = false;
+            if (!alive) continue;                                       // keep arriving at the named barrier above
+            const uint32_t xs = sbase + s * L::kStage + L::kWStage;
+#pragma unroll
+            for (int tb = 0; tb < L::kTokBlocks; ++tb) {
+                const int local = tb * 64 + cc * 8;                       // token index inside this CTA's half
+                if (local < L::kHalf) {
+                    const int t = tok_cta + local;
+                    const int valid = min(8, max(0, p.M - t));
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int r = rg + 64 * i;
+                        const bool in = ch[i] >= 0 && valid > 0;
+                        const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
+                        cp_async_16(xs + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4), src, in ? valid * 2 : 0);
+                    }
+                }
+            }
+            cp_async_arrive_noinc(full(s));
+        }
+        // ---- epilogue: this CTA's 128 feature rows of every accumulator, all TN token columns; warp w reads lane
+        // quarter w % 4 and the 16-column pieces (w - 2) / 4, + 4, + 8, ...
+        const int quarter = warp & 3;
+        const int cgrp = (warp - 2) >> 2;
+        const int f_local = quarter * 32 + lane;
+        const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait_cluster(accum_bar, 0, abort_flag)));
+        tc_fence_after();
+        const int esize = p.out_f32 ? 4 : 2;
+        const int row_bytes = 128 * esize;
+        const int chunks_per_row = row_bytes / 16;
+        const bool vec_ok = (((long)p.ldy * esize) % 16 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0);
+        uint8_t *yb = reinterpret_cast<uint8_t *>(p.Y);
+#pragma unroll 1
+        for (int a = 0; a < NA; ++a) {
+            if (a > 0) asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");   // the staging area is free again
+#pragma unroll 1
+            for (int c0 = cgrp * 16; c0 < TN; c0 += 64) {
+                uint32_t v[16];
+                if (nk > 0 && ok) {
+                    tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + L::acc_col(a) + c0, v);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0;
+                }
+                if (p.out_f32) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
+                }
+            }
+            tc_fence_before();
+            asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");
+            if (!present[a]) continue;
+            const int f_valid = min(128, p.N - ftile[a] * 128);
+            for (int idx = g; idx < TN * chunks_per_row; idx += kPairProducers) {
+                const int row = idx / chunks_per_row, c = idx % chunks_per_row;
+                const int t = tok0 + row;
+                if (!ok || t >= p.M) continue;
+                const int f0 = c * (16 / esize);
+                uint8_t *dst = yb + ((long)t * p.ldy + (long)ftile[a] * 128 + f0) * esize;
+                const uint8_t *srcp = smem + (size_t)row * row_bytes + c * 16;
+                if (vec_ok && f0 + 16 / esize <= f_valid) {
+                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(srcp);
+                } else {
+                    for (int e = 0; e < 16 / esize; ++e)
+                        if (f0 + e < f_valid) {
+                            if (p.out_f32) reinterpret_cast<float *>(dst)[e] = reinterpret_cast<const float *>(srcp)[e];
+                            else reinterpret_cast<uint16_t *>(dst)[e] = reinterpret_cast<const uint16_t *>(srcp)[e];
+                        }
+                }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    cluster_sync_all();                      // both CTAs are done with tensor memory and with each other's barriers
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem, L::kTmemCols);
+    }
+}
+
+template <int NA, int TN>
+esp_status_t launch_pair(const GemmParams &p, cudaStream_t stream) {
+    using L = PairCfg<NA, TN>;
+    auto kern = spgemm_pair_kernel<NA, TN>;
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    const int f_tiles = (p.N + 127) / 128;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ((f_tiles + 2 * NA - 1) / (2 * NA)), (p.M + TN - 1) / TN, 1);
+    cfg.blockDim = dim3(kPairThreads);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
+    return ESP_OK;
+}

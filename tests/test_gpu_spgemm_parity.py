@@ -94,6 +94,34 @@ def test_prefill_tiled_kernels(M, N, K, kernel):
           orc.product(X, vals, meta, None))
 
 
+@pytest.mark.parametrize("M", [130, 300, 520, 1000])
+@pytest.mark.parametrize("N,K", [(256, 512), (200, 264), (640, 1160), (1100, 384)])
+def test_prefill_pair_kernel(M, N, K):
+    """The two-SM kernel (5): feature-pair tiles with one to four of their 128-feature tiles present, ragged
+    token / feature / channel tails, every tile width, both layouts and output types."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(N * 5 + K + M, N, K)
+    X = np.random.default_rng(M + 2).standard_normal((M, K)).astype(np.float16)
+    Yref = orc.product(X, vals, meta, theta)
+    packed = pack_on_gpu(vals, meta)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=5), Yref)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=5, out_f32=True), Yref, True)
+    for tile in (128, 192, 224, 256):
+        check(spgemm(X, packed, theta, N, channel_major=True, kernel=5, token_tile=tile, out_f32=True), Yref, True)
+    check(spgemm(X, packed, theta, N, kernel=5), Yref)                          # token-major via the transposed copy
+    check(spgemm(X, packed, None, N, channel_major=True, kernel=5), orc.product(X, vals, meta, None))
+
+
+def test_pair_kernel_long_k_and_determinism():
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(13, 384, 4224)                                  # 33 channel tiles > the permutation ring
+    packed = pack_on_gpu(vals, meta)
+    X = np.random.default_rng(5).standard_normal((500, 4224)).astype(np.float16)
+    a = spgemm(X, packed, theta, 384, channel_major=True, kernel=5, out_f32=True)
+    assert np.array_equal(a, spgemm(X, packed, theta, 384, channel_major=True, kernel=5, out_f32=True))
+    check(a, orc.product(X, vals, meta, theta), True)
+
+
 def test_identity_permutation_and_unit_rows():
     """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
     from tests.gpu_util import pack_on_gpu, spgemm
