@@ -729,15 +729,19 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
         mbar_init(recv_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
-        // the weight stream starts now: nothing below is needed for these copies
-        for (int it = 0; it < prefetch; ++it) {
-            mbar_arrive_expect_tx(full(it), kTileBytes);
-            bulk_load(sbase + it * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(it));
-        }
         if (L::kPush && split > 1) {
             // every sender delivers 128 features x (rows of this tile that this CTA owns) floats
             const int owned = (BN - (int)rank + split - 1) / split;
             mbar_arrive_expect_tx(recv_bar, (uint32_t)(split * owned * 512));
+        }
+    }
+    if (warp == 0) {
+        // The weight stream starts now: nothing below is needed for these copies.  Lane s owns stage s (bulk copies
+        // issued by one thread complete one after the other, copies of different threads overlap).
+        __syncwarp();
+        if (lane < prefetch) {
+            mbar_arrive_expect_tx(full(lane), kTileBytes);
+            bulk_load(sbase + lane * L::kStage, w_src + (long)lane * kTileBytes, kTileBytes, full(lane));
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
@@ -761,13 +765,12 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
     grid_launch_dependents();
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int it = prefetch; it < nk; ++it) {
-                const int s = it % stages;
+        if (lane < stages) {
+            for (int it = lane + stages; it < nk; it += stages) {      // this lane's stage, every later round
                 const uint32_t ph = (uint32_t)(it / stages) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
-                mbar_arrive_expect_tx(full(s), kTileBytes);
-                bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
+                if (!mbar_wait(empty(lane), ph ^ 1u, abort_flag)) break;
+                mbar_arrive_expect_tx(full(lane), kTileBytes);
+                bulk_load(sbase + lane * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(lane));
             }
         }
         __syncwarp();

@@ -22,7 +22,7 @@
 //     512, independent of how many stages are in flight, so sixteen warps gather X.
 //
 // grid (2 x feature-pair tiles, token tiles, 1), cluster (2,1,1), block 576.  In both CTAs:
-//   warp 0 lanes 0..3  weight-tile producers (tile copies dealt round-robin)
+//   warp 0             weight-tile producers (one lane per stage and feature tile)
 //   warp 1             tensor-memory allocation; lane 0 of the leader CTA (rank 0): tcgen05.cp + MMAs for the pair;
 //                      lane 0 of rank 1: forwards "my stage is full" to the leader's barrier
 //   warps 2..17        X row producers, then epilogue (four warps per quarter of the accumulator lanes)
@@ -57,7 +57,6 @@ __device__ __forceinline__ void tc_mma_sparse_f16_pair(uint32_t d_tmem, uint64_t
 
 constexpr int kPairProducers = 512;                  // X producer threads (warps 2..17)
 constexpr int kPairThreads = 64 + kPairProducers;
-constexpr int kPairIssuers = 4;                      // lanes of warp 0 that issue weight-tile copies
 
 template <int NA, int TN>
 struct PairCfg {
@@ -151,11 +150,12 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
-        if (lane < kPairIssuers) {
-            // copy number q = it * NA + a goes to lane q % kPairIssuers (copies of one thread do not overlap)
-            for (int q = lane; q < nk * NA; q += kPairIssuers) {
-                const int it = q / NA, a = q % NA;
-                if (!present[a]) continue;
+        if (lane < NA * STAGES) {
+            // copies of one thread do not overlap, so tile a of stage s has its own lane s * NA + a; a lane then meets
+            // its stage's barriers in every phase (a parity wait cannot tell phases two apart)
+            const int a = lane % NA;
+            for (int it = lane / NA; it < nk; it += STAGES) {
+                if (!present[a]) break;
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                 if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
