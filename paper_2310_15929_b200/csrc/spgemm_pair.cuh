@@ -22,10 +22,11 @@
 //     512, independent of how many stages are in flight, so sixteen warps gather X.
 //
 // grid (2 x feature-pair tiles, token tiles, 1), cluster (2,1,1), block 576.  In both CTAs:
-//   warp 0             weight-tile producers (one lane per stage and feature tile)
+//   warp 0             idle
 //   warp 1             tensor-memory allocation; lane 0 of the leader CTA (rank 0): tcgen05.cp + MMAs for the pair;
 //                      lane 0 of rank 1: forwards "my stage is full" to the leader's barrier
-//   warps 2..17        X row producers, then epilogue (four warps per quarter of the accumulator lanes)
+//   warps 2..17        X row producers (lane 0 of six of them also issues the weight-tile copies), then epilogue
+//                      (four warps per quarter of the accumulator lanes)
 // A stage's `empty` barrier and the final `accum` barrier are signalled in both CTAs at once by
 // tcgen05.commit with a CTA mask.  No load uses cluster multicast.
 
@@ -65,10 +66,9 @@ struct PairCfg {
     static constexpr int kXStage = kTokBlocks * 16384;
     static constexpr int kWStage = NA * kTileBytes;
     static constexpr int kStage = kWStage + kXStage;                  // a multiple of 1024
-    static constexpr int kStagesFit = (227 * 1024 - kPermRing * 512 - 512 - 1024) / kStage;
+    static constexpr int kStagesFit = (227 * 1024 - 512 - 1024) / kStage;
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
-    static constexpr int kPermOff = kStages * kStage;
-    static constexpr int kBarOff = kPermOff + kPermRing * 512;
+    static constexpr int kBarOff = kStages * kStage;
     static constexpr int kTotal = kBarOff + 512 + 1024;
     static constexpr uint32_t kTmemCols = 512;
     static_assert(NA * 256 <= 512 && TN + 8 <= 256 + (NA == 1 ? 8 : 0) && TN % 16 == 0, "tensor memory layout");
@@ -90,7 +90,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const uint32_t accum_bar = bar_base + 8u * 24;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
-    int *perm_s = reinterpret_cast<int *>(smem + L::kPermOff);           // [kPermRing][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                              // 0 = leader
@@ -130,19 +129,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             }
         }
     }
-    if (warp >= 2) {
-        // permutation entries of the first kPermRing stages: thread g takes row g % 128 of stages g / 128 + 4 i
-        const int g = threadIdx.x - 64;
-        int pre[kPermRing / 4];
-#pragma unroll
-        for (int i = 0; i < kPermRing / 4; ++i) {
-            const int it = (g >> 7) + 4 * i;
-            const int kpos = it * kTileK + (g & 127);
-            pre[i] = (it < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
-        }
-#pragma unroll
-        for (int i = 0; i < kPermRing / 4; ++i) perm_s[((g >> 7) + 4 * i) * 128 + (g & 127)] = pre[i];
-    }
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();                      // both CTAs have their barriers and tensor memory before any cross-CTA signal
@@ -150,20 +136,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
-        if (lane < NA * STAGES) {
-            // copies of one thread do not overlap, so tile a of stage s has its own lane s * NA + a; a lane then meets
-            // its stage's barriers in every phase (a parity wait cannot tell phases two apart)
-            const int a = lane % NA;
-            for (int it = lane / NA; it < nk; it += STAGES) {
-                if (!present[a]) break;
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) break;
-                mbar_arrive_expect_tx(full(s), kTileBytes);
-                bulk_load(sbase + s * L::kStage + a * kTileBytes, p.packed + ((long)ftile[a] * p.k_tiles + it) * kTileBytes,
-                          kTileBytes, full(s));
-            }
-        }
+        // idle: keeps the producer warps at indices 2..17 (tensor-memory lane quarter = warp index % 4)
     } else if (warp == 1) {
         if (lane == 0 && rank != 0) {
             // forward "my operands of this stage have landed" to the leader
@@ -175,76 +148,107 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 mbar_arrive_remote(map_to_rank(peer_full(s), 0));
             }
         } else if (lane == 0) {
+            // One thread issues every MMA of the pair, so its own instruction stream must stay far shorter than the
+            // MMAs' execution time: all descriptors are built once (stage 0) and a stage only adds its byte offset
+            // (>> 4) to their low words; the loop is unrolled over the ring and the metadata double buffer so that
+            // every column index and offset is a compile-time constant.
             constexpr uint32_t idesc = instr_desc_sparse_f16(256, TN, 1);
-            for (int it = 0; it < nk; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                if (!mbar_wait(full(s), ph, abort_flag)) break;
-                if (!mbar_wait_cluster(peer_full(s), ph, abort_flag)) break;
-                fence_async_smem();
-                tc_fence_after();
-                const uint32_t wa = sbase + s * L::kStage;
-                const uint32_t xa = wa + L::kWStage;
+            uint64_t ad0[NA][4], bd0[4], md0[NA];
 #pragma unroll
-                for (int a = 0; a < NA; ++a) {
-                    const uint32_t e_col = L::meta_col(a, it & 1);
-                    const uint32_t ta = wa + a * kTileBytes;
-                    tc_copy_128x128b_pair(tmem + e_col, smem_desc(ta + kTileValBytes, 0, 128, kLayoutNone));
+            for (int a = 0; a < NA; ++a) {
+                md0[a] = smem_desc(sbase + a * kTileBytes + kTileValBytes, 0, 128, kLayoutNone);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t col = e_col + j;
-                        const uint64_t ad = smem_desc(ta + j * 32, 16, 1024, kLayoutSw128);
-                        const uint64_t bd = smem_desc(xa + j * 4096, 16384, 1024, kLayoutSw128);
-                        tc_mma_sparse_f16_pair(tmem + L::acc_col(a), ad, bd, tmem + (col & ~1u), idesc | (col & 1u),
-                                               (it > 0 || j > 0) ? 1u : 0u);
+                for (int j = 0; j < 4; ++j) ad0[a][j] = smem_desc(sbase + a * kTileBytes + j * 32, 16, 1024, kLayoutSw128);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bd0[j] = smem_desc(sbase + L::kWStage + j * 4096, 16384, 1024, kLayoutSw128);
+            constexpr int kUnroll = STAGES * 2;                           // ring slot and metadata buffer both periodic
+            bool alive = true;
+            for (int it0 = 0; it0 < nk && alive; it0 += kUnroll) {
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const int it = it0 + u;
+                    if (it >= nk) break;
+                    const int s = u % STAGES;                             // == it % STAGES (it0 is a multiple of STAGES)
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(full(s), ph, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait_cluster(peer_full(s), ph, abort_flag)) { alive = false; break; }
+                    fence_async_smem();
+                    tc_fence_after();
+                    const uint64_t soff = (uint64_t)((uint32_t)(s * L::kStage) >> 4);   // added to the address field
+#pragma unroll
+                    for (int a = 0; a < NA; ++a) {
+                        const uint32_t e_col = L::meta_col(a, u & 1);     // == meta_col(a, it & 1) (kUnroll is even)
+                        tc_copy_128x128b_pair(tmem + e_col, md0[a] + soff);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t col = e_col + j;
+                            tc_mma_sparse_f16_pair(tmem + L::acc_col(a), ad0[a][j] + soff, bd0[j] + soff, tmem + (col & ~1u),
+                                                   idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
+                        }
                     }
+                    tc_commit_pair(empty(s), (uint16_t)3);
                 }
-                tc_commit_pair(empty(s), (uint16_t)3);
             }
             tc_commit_pair(accum_bar, (uint16_t)3);
         }
     } else {
-        // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) and (g >> 3) + 64 of every 64-token block
+        // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) and (g >> 3) + 64 of every 64-token
+        // block.  Its two permutation entries are loaded kAhead steps early into registers (the loop is unrolled by
+        // kAhead so the register ring has constant indices): the load's latency never sits between two steps.
         const int g = threadIdx.x - 64;
         const int cc = g & 7, rg = g >> 3;
         const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
-        const bool ring_refill = nk > kPermRing;
         bool alive = true;
-        int refill = -1;
-        for (int it = 0; it < nk; ++it) {
-            const int s = it % STAGES;
-            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-            const int *pr = perm_s + (it % kPermRing) * 128;
-            if (ring_refill && it > 0 && g < 128) perm_s[((it - 1) % kPermRing) * 128 + g] = refill;   // stage it-1+kPermRing
-            int ch[2];
-            ch[0] = pr[rg];
-            ch[1] = pr[rg + 64];
-            if (ring_refill) {
-                asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");   // everyone has read this stage's entries
-                if (g < 128) {
-                    const int kpos = (it + kPermRing) * kTileK + g;
-                    refill = (it + kPermRing < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+        constexpr int kAhead = 4;
+        auto channel_of = [&](int it, int row) -> int {
+            const int kpos = it * kTileK + row;
+            return (it < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+        };
+        int nxt[kAhead][2];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) { nxt[u][0] = channel_of(u, rg); nxt[u][1] = channel_of(u, rg + 64); }
+        for (int it0 = 0; it0 < nk; it0 += kAhead) {
+#pragma unroll
+            for (int u = 0; u < kAhead; ++u) {
+                const int it = it0 + u;
+                if (it >= nk) break;
+                const int ch[2] = {nxt[u][0], nxt[u][1]};
+                nxt[u][0] = channel_of(it + kAhead, rg);
+                nxt[u][1] = channel_of(it + kAhead, rg + 64);
+                const int s = it % STAGES;
+                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                if (alive && !mbar_wait(empty(s), ph ^ 1u, abort_flag)) alive = false;
+                if (!alive) continue;
+                const uint32_t xs = sbase + s * L::kStage + L::kWStage;
+#pragma unroll
+                for (int tb = 0; tb < L::kTokBlocks; ++tb) {
+                    const int local = tb * 64 + cc * 8;                   // token index inside this CTA's half
+                    if (local < L::kHalf) {
+                        const int t = tok_cta + local;
+                        const int valid = min(8, max(0, p.M - t));
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            const int r = rg + 64 * i;
+                            const bool in = ch[i] >= 0 && valid > 0;
+                            const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
+                            cp_async_16(xs + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4), src, in ? valid * 2 : 0);
+                        }
+                    }
                 }
-            }
-            if (alive && !mbar_wait(empty(s), ph ^ 1u, abort_flag)) alive = false;
-            if (!alive) continue;                                       // keep arriving at the named barrier above
-            const uint32_t xs = sbase + s * L::kStage + L::kWStage;
-#pragma unroll
-            for (int tb = 0; tb < L::kTokBlocks; ++tb) {
-                const int local = tb * 64 + cc * 8;                       // token index inside this CTA's half
-                if (local < L::kHalf) {
-                    const int t = tok_cta + local;
-                    const int valid = min(8, max(0, p.M - t));
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const int r = rg + 64 * i;
-                        const bool in = ch[i] >= 0 && valid > 0;
-                        const uint16_t *src = in ? xb + (long)ch[i] * p.ldx + t : xb;
-                        cp_async_16(xs + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4), src, in ? valid * 2 : 0);
+                cp_async_arrive_noinc(full(s));
+                // Weight tile a of this stage is issued by lane 0 of producer warp s * NA + a: copies issued by one thread
+                // do not overlap, and spinning lanes of one warp would hold each other up, so every copy of the ring
+                // has a warp of its own, which has just seen the stage's `empty` barrier anyway.
+                if (lane == 0 && (warp - 2) / NA == s && (warp - 2) < NA * STAGES) {
+                    const int a = (warp - 2) % NA;
+                    if (present[a]) {
+                        mbar_arrive_expect_tx(full(s), kTileBytes);
+                        bulk_load(sbase + s * L::kStage + a * kTileBytes,
+                                  p.packed + ((long)ftile[a] * p.k_tiles + it) * kTileBytes, kTileBytes, full(s));
                     }
                 }
             }
-            cp_async_arrive_noinc(full(s));
         }
         // ---- epilogue: this CTA's 128 feature rows of every accumulator, all TN token columns; warp w reads lane
         // quarter w % 4 and the 16-column pieces (w - 2) / 4, + 4, + 8, ...
