@@ -56,6 +56,28 @@ __device__ __forceinline__ void tc_mma_sparse_f16_pair(uint32_t d_tmem, uint64_t
         : "memory");
 }
 
+// Waits of the two single-thread roles (forwarder, MMA issuer), each alone in its warp: poll without sleeping first --
+// a sleeping poll adds its sleep to every hand-over of the ring -- then fall back to the bounded, abort-aware wait.
+__device__ __forceinline__ bool mbar_wait_1t(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < (1u << 15); ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity, abort_flag);
+}
+__device__ __forceinline__ bool mbar_wait_cluster_1t(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < (1u << 15); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return mbar_wait_cluster(bar, parity, abort_flag);
+}
+
 constexpr int kPairProducers = 512;                  // X producer threads (warps 2..17)
 constexpr int kPairThreads = 64 + kPairProducers;
 
@@ -143,7 +165,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             for (int it = 0; it < nk; ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                if (!mbar_wait(full(s), ph, abort_flag)) break;
+                if (!mbar_wait_1t(full(s), ph, abort_flag)) break;
                 fence_async_smem();          // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
                 mbar_arrive_remote(map_to_rank(peer_full(s), 0));
             }
@@ -171,8 +193,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                     if (it >= nk) break;
                     const int s = u % STAGES;                             // == it % STAGES (it0 is a multiple of STAGES)
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                    if (!mbar_wait(full(s), ph, abort_flag)) { alive = false; break; }
-                    if (!mbar_wait_cluster(peer_full(s), ph, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait_1t(full(s), ph, abort_flag)) { alive = false; break; }
+                    if (!mbar_wait_cluster_1t(peer_full(s), ph, abort_flag)) { alive = false; break; }
                     fence_async_smem();
                     tc_fence_after();
                     const uint64_t soff = (uint64_t)((uint32_t)(s * L::kStage) >> 4);   // added to the address field
@@ -257,14 +279,11 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         const int f_local = quarter * 32 + lane;
         const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait_cluster(accum_bar, 0, abort_flag)));
         tc_fence_after();
-        const int esize = p.out_f32 ? 4 : 2;
-        const int row_bytes = 128 * esize;
-        const int chunks_per_row = row_bytes / 16;
-        const bool vec_ok = (((long)p.ldy * esize) % 16 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0);
-        uint8_t *yb = reinterpret_cast<uint8_t *>(p.Y);
-#pragma unroll 1
-        for (int a = 0; a < NA; ++a) {
-            if (a > 0) asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");   // the staging area is free again
+        const bool y_vec = (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
+        // accumulator a -> shared memory [token][128 features] in the output type -> 16-byte stores along the features.
+        // fp16 output: both accumulators are staged side by side (2 x TN x 256 bytes) and stored in one sweep.
+        auto stage_acc = [&](int a, uint8_t *area, auto out_tag) {
+            using OutT = decltype(out_tag);
 #pragma unroll 1
             for (int c0 = cgrp * 16; c0 < TN; c0 += 64) {
                 uint32_t v[16];
@@ -274,34 +293,51 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 #pragma unroll
                     for (int e = 0; e < 16; ++e) v[e] = 0;
                 }
-                if (p.out_f32) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
+                for (int e = 0; e < 16; ++e) {
+                    if (sizeof(OutT) == 4) reinterpret_cast<float *>(area)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+                    else reinterpret_cast<__half *>(area)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
                 }
             }
-            tc_fence_before();
-            asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");
-            if (!present[a]) continue;
+        };
+        auto store_acc = [&](int a, const uint8_t *area, auto out_tag) {
+            using OutT = decltype(out_tag);
+            constexpr int kPer = 16 / (int)sizeof(OutT);                  // features per 16-byte piece
+            constexpr int kPieces = 128 / kPer;                           // pieces per token row
+            if (!present[a]) return;
             const int f_valid = min(128, p.N - ftile[a] * 128);
-            for (int idx = g; idx < TN * chunks_per_row; idx += kPairProducers) {
-                const int row = idx / chunks_per_row, c = idx % chunks_per_row;
+            const bool vec_ok = y_vec && (((long)p.ldy * (long)sizeof(OutT)) % 16 == 0);
+            OutT *yo = reinterpret_cast<OutT *>(p.Y) + (long)ftile[a] * 128;
+            for (int idx = g; idx < TN * kPieces; idx += kPairProducers) {
+                const int row = idx / kPieces, c = idx % kPieces;
                 const int t = tok0 + row;
                 if (!ok || t >= p.M) continue;
-                const int f0 = c * (16 / esize);
-                uint8_t *dst = yb + ((long)t * p.ldy + (long)ftile[a] * 128 + f0) * esize;
-                const uint8_t *srcp = smem + (size_t)row * row_bytes + c * 16;
-                if (vec_ok && f0 + 16 / esize <= f_valid) {
+                const int f0 = c * kPer;
+                OutT *dst = yo + (long)t * p.ldy + f0;
+                const OutT *srcp = reinterpret_cast<const OutT *>(area) + row * 128 + f0;
+                if (vec_ok && f0 + kPer <= f_valid) {
                     *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(srcp);
                 } else {
-                    for (int e = 0; e < 16 / esize; ++e)
-                        if (f0 + e < f_valid) {
-                            if (p.out_f32) reinterpret_cast<float *>(dst)[e] = reinterpret_cast<const float *>(srcp)[e];
-                            else reinterpret_cast<uint16_t *>(dst)[e] = reinterpret_cast<const uint16_t *>(srcp)[e];
-                        }
+                    for (int e = 0; e < kPer; ++e)
+                        if (f0 + e < f_valid) dst[e] = srcp[e];
                 }
+            }
+        };
+        if (!p.out_f32) {
+#pragma unroll 1
+            for (int a = 0; a < NA; ++a) stage_acc(a, smem + (size_t)a * TN * 256, __half());
+            tc_fence_before();
+            asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");
+#pragma unroll 1
+            for (int a = 0; a < NA; ++a) store_acc(a, smem + (size_t)a * TN * 256, __half());
+        } else {
+#pragma unroll 1
+            for (int a = 0; a < NA; ++a) {
+                if (a > 0) asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");   // the staging area is free again
+                stage_acc(a, smem, float());
+                tc_fence_before();
+                asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");
+                store_acc(a, smem, float());
             }
         }
         tc_fence_before();
