@@ -66,6 +66,10 @@ typedef struct {
     int use_gns;                 /* 0 skips the global naive shuffle (identity start order)           */
     int use_lbs;                 /* 0 skips the local block shuffle                                   */
     const double *score_override;/* optional device f64[C]: use these s_c instead of computing them   */
+    const int32_t *perm_override;/* optional device i32[C]: start from this channel order instead of the
+                                    global shuffle's (a stored permutation, e.g. to re-compress updated
+                                    weights); the block shuffle still runs on it if use_lbs is set.
+                                    Must be a permutation of 0..C-1 (not checked).                     */
 } esp_prune_opts;
 
 typedef struct {

@@ -24,7 +24,8 @@ ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNE
 class esp_prune_opts(ctypes.Structure):
     _fields_ = [("struct_size", c_size_t), ("alpha", c_double), ("bins", c_int), ("n_keep", c_int),
                 ("m_group", c_int), ("lbs_block", c_int), ("lbs_max_swaps", c_int), ("use_entropy", c_int),
-                ("use_norm", c_int), ("use_gns", c_int), ("use_lbs", c_int), ("score_override", c_void_p)]
+                ("use_norm", c_int), ("use_gns", c_int), ("use_lbs", c_int), ("score_override", c_void_p),
+                ("perm_override", c_void_p)]
 
 
 class esp_prune_stats(ctypes.Structure):

@@ -86,6 +86,7 @@ void esp_prune_opts_default(esp_prune_opts *o) {
     o->use_gns = 1;
     o->use_lbs = 1;
     o->score_override = nullptr;
+    o->perm_override = nullptr;
 }
 
 void esp_gemm_opts_default(esp_gemm_opts *o) {

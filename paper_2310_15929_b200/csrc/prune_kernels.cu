@@ -681,14 +681,17 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     if (chan_score) ESP_CUDA_OK(cudaMemcpyAsync(chan_score, w.score, sizeof(double) * C, cudaMemcpyDeviceToDevice, stream));
 
     // K3 + K4
-    if (o.use_gns) {
+    if (o.use_gns && !o.perm_override) {
         ESP_CUDA_OK(cudaMemsetAsync(w.colsum, 0, sizeof(unsigned long long) * C, stream));
         const int wsplits = pick_splits(No, ceil_div(C, 256), di.sm_count);
         colabs_kernel<<<dim3(ceil_div(C, 256), wsplits), 256, 0, stream>>>(W, No, C, ldw, ceil_div(No, wsplits), w.colsum);
         mean_metric_kernel<<<cblocks, cthreads, 0, stream>>>(C, No, w.colsum, w.score, w.mean);
     }
     int32_t *theta0 = (o.use_lbs || stats) ? w.theta0 : perm;
-    gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, theta0);
+    if (o.perm_override)
+        ESP_CUDA_OK(cudaMemcpyAsync(theta0, o.perm_override, sizeof(int32_t) * C, cudaMemcpyDeviceToDevice, stream));
+    else
+        gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, theta0);
     ESP_CUDA_OK(cudaGetLastError());
 
     // K5

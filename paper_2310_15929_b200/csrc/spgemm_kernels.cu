@@ -1160,7 +1160,16 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
         else g.kernel = (M > 256 && o.split_k <= 1) ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;   // the pair kernel has no K-slices
     }
     if (g.kernel == ESP_KERNEL_PAIR) {
-        if (bn == 0) bn = 240;
+        if (bn == 0) {
+            // widest token tile unless a narrower one saves a whole wave of clusters: cost ~ waves x tile width
+            const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
+            long best = -1;
+            for (int tn : {240, 224, 192}) {
+                const long clusters = f_pairs * ceil_div(M, tn);
+                const long cost = ceil_div(clusters, per_wave) * tn;
+                if (best < 0 || cost < best) { best = cost; bn = tn; }
+            }
+        }
         if (bn != 128 && bn != 192 && bn != 224 && bn != 240 && bn != 256) return ESP_ERR_INVALID_ARG;
         g.token_tile = bn;
         g.split_k = 1;

@@ -10,7 +10,7 @@ DEV = "cuda:0"
 
 
 class GpuPrune:
-    def __init__(self, W, Xcal, alpha, score=None, stats=True, pack=True, **opts):
+    def __init__(self, W, Xcal, alpha, score=None, stats=True, pack=True, perm=None, **opts):
         No, C = W.shape
         self.No, self.C = No, C
         dev = torch.device(DEV)
@@ -25,6 +25,10 @@ class GpuPrune:
         if score is not None:
             self.score_d = torch.from_numpy(np.ascontiguousarray(score, dtype=np.float64)).to(dev)
             o.score_override = self.score_d.data_ptr()
+        self.perm_in = None
+        if perm is not None:
+            self.perm_in = torch.from_numpy(np.ascontiguousarray(perm, dtype=np.int32)).to(dev)
+            o.perm_override = self.perm_in.data_ptr()
         self.ws = torch.empty(max(16, b.esp_metric_prune_workspace_bytes(No, C, T, o)), dtype=torch.uint8, device=dev)
         self.vals = torch.empty(No, C // 2, dtype=torch.float16, device=dev)
         self.meta = torch.empty(No, C // 8, dtype=torch.uint8, device=dev)
