@@ -101,6 +101,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(x, dist, device):
+    """The largest of one float per rank (every rank gets it).  dist = torch.distributed or None for one rank."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(work_per_rank, world, ms_max):
+    """Aggregate rate of `world` replicas that each did `work_per_rank` while the slowest took ms_max."""
+    return world * work_per_rank / (ms_max * 1e-3)
+
+
 def gemm_bytes(M, N, K):
     """Algorithmic bytes of one sparse GEMM: compressed weight + metadata, X, Y, permutation."""
     return 1.125 * N * K + 2.0 * M * K + 2.0 * M * N + 4.0 * K
@@ -275,13 +290,11 @@ def run_ours(args):
     torch.cuda.synchronize()
     clocks = sampler.stop(t_begin)
     clocks["covers"] = f"the {args.steps} timed steps and {extra_steps} further identical steps"
+    ms = max_over_ranks(ms, dist, dev)
     if dist:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
         dist.barrier()
     flops = sum(2.0 * PREFILL_M * lin["N"] * lin["K"] for lin in layer)
-    value = world * flops / (ms * 1e-3) / 1e12
+    value = whole_job_rate(flops, world, ms) / 1e12
     assert b.esp_last_device_status() == b.ESP_OK
 
     # ---------------- end to end through the C ABI with host buffers ----------------
@@ -296,11 +309,8 @@ def run_ours(args):
             b.esp_spgemm(X, lin["packed"], lin["perm"], Y, po, pws)
             HY.copy_(Y, non_blocking=True)
     e2e_ms = time_steps(e2e_step, max(2, args.steps // 4), 2)
-    if dist:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    e2e = {"value": whole_job_rate(flops, world, e2e_ms) / 1e12, "unit": "TFLOP/s",
            "h2d_bytes_per_step": int(sum(h.numel() * 2 for h in hx)),
            "d2h_bytes_per_step": int(sum(h.numel() * 2 for h in hy))}
 
