@@ -311,13 +311,124 @@ __device__ double group_value_warp(const uint16_t *__restrict__ Wt, long ldt, co
     return __dadd_rn(__dadd_rn(__dadd_rn(t0, t1), t2), t3);
 }
 
+// --------------------------------------------------------------------------------------------------
+// V(group with slot k replaced by candidate x) for all candidates x of a block, without re-ranking four columns
+// per row and candidate.  With the three fixed slots ordered f1, f2, f3 by the metric (ties: lower slot), the
+// candidate is kept exactly when it is ahead of f2; f1 is always kept, f2 is kept exactly when the candidate is not,
+// f3 never.  So per row only f2's slot and |w| matter: phase 1 stores them (4 bytes per row, shared memory) and the
+// exact sums B_q of |w_q| over rows where q is f1 or f2; phase 2 (one warp per candidate) needs one multiply and one
+// compare per row and candidate:  A_x = sum kept |w_x|,  A_q = B_q - sum [q is f2 and x kept] |w_q|.
+// The kept sets, the exact integer sums and the order of the four multiplies and three adds are those of
+// group_value_warp, so the values are bit-identical to it.
+// --------------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool metric_ahead(double xa, int sa, double xb, int sb) { return xa > xb || (xa == xb && sa < sb); }
+
+// Phase 1, whole CTA.  ch[4]: the group's channels; k: the slot to be replaced.  pk[j] = f2 slot << 16 | |w_f2| bits.
+// s_B[4] (shared, zeroed by the caller before the preceding barrier) receives B_q.
+__device__ void lbs_slot_prepare(const uint16_t *__restrict__ Wt, long ldt, const double *__restrict__ score,
+                                 const int (&ch)[4], int k, uint32_t *__restrict__ pk, unsigned long long *s_B) {
+    double sc[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) sc[q] = score[ch[q]];
+    long long B[4] = {0, 0, 0, 0};
+    for (long j = (long)threadIdx.x * 8; j < ldt; j += (long)blockDim.x * 8) {
+        uint4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (q != k) v[q] = *reinterpret_cast<const uint4 *>(Wt + (long)ch[q] * ldt + j);
+        uint32_t out[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            uint16_t h[4];
+            double xi[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                h[q] = (q != k) ? reinterpret_cast<const uint16_t *>(&v[q])[e] : (uint16_t)0;
+                xi[q] = __dmul_rn(half_bits_abs_to_double(h[q]), sc[q]);
+            }
+            // rank of each fixed slot among the three fixed ones
+            int f1 = -1, f2 = -1;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q == k) continue;
+                int ahead = 0;
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    if (r != k && r != q) ahead += metric_ahead(xi[r], r, xi[q], q) ? 1 : 0;
+                if (ahead == 0) f1 = q;
+                if (ahead == 1) f2 = q;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (q == f1 || q == f2) B[q] += half_bits_abs_fixed(h[q]);
+            uint16_t hf2 = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (q == f2) hf2 = h[q];
+            out[e] = ((uint32_t)f2 << 16) | hf2;
+        }
+        *reinterpret_cast<uint4 *>(pk + j) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4 *>(pk + j + 4) = make_uint4(out[4], out[5], out[6], out[7]);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) B[q] += __shfl_xor_sync(0xFFFFFFFFu, B[q], off);
+        if ((threadIdx.x & 31) == 0 && B[q]) atomicAdd(&s_B[q], (unsigned long long)B[q]);   // integers: order-free
+    }
+}
+
+// Phase 2, one warp: the value for candidate channel cx in slot k.  Every lane returns it.
+__device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, const double (&sc_fixed)[4], int k, int cx,
+                                     double sx, const uint32_t *__restrict__ pk, const unsigned long long *s_B) {
+    const int lane = threadIdx.x & 31;
+    long long Ax = 0, D[4] = {0, 0, 0, 0};
+    for (long j = lane * 8; j < ldt; j += 256) {
+        const uint4 vx = *reinterpret_cast<const uint4 *>(Wt + (long)cx * ldt + j);
+        const uint4 p0 = *reinterpret_cast<const uint4 *>(pk + j);
+        const uint4 p1 = *reinterpret_cast<const uint4 *>(pk + j + 4);
+        const uint32_t pkv[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint16_t hx = reinterpret_cast<const uint16_t *>(&vx)[e];
+            const int f2 = (int)(pkv[e] >> 16);
+            const uint16_t hf = (uint16_t)(pkv[e] & 0xFFFFu);
+            const double sf = f2 == 0 ? sc_fixed[0] : f2 == 1 ? sc_fixed[1] : f2 == 2 ? sc_fixed[2] : sc_fixed[3];
+            const double xx = __dmul_rn(half_bits_abs_to_double(hx), sx);
+            const double xf = __dmul_rn(half_bits_abs_to_double(hf), sf);
+            const bool kept = metric_ahead(xx, k, xf, f2);
+            const long long wf = kept ? half_bits_abs_fixed(hf) : 0;
+            Ax += kept ? half_bits_abs_fixed(hx) : 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) D[q] += (q == f2) ? wf : 0;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        Ax += __shfl_xor_sync(0xFFFFFFFFu, Ax, off);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) D[q] += __shfl_xor_sync(0xFFFFFFFFu, D[q], off);
+    }
+    double t[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const long long A = (q == k) ? Ax : (long long)s_B[q] - D[q];
+        const double sq = (q == k) ? sx : sc_fixed[q];
+        t[q] = __dmul_rn(sq, __dmul_rn(__ll2double_rn(A), 0x1p-24));
+    }
+    return __dadd_rn(__dadd_rn(__dadd_rn(t[0], t[1]), t[2]), t[3]);
+}
+
 // table[b][g][slot][x] = V(group g of block b with its slot replaced by block channel x); base[G] = V(g).
-// grid (nblocks * 64), block 256 (8 warps).
+// grid (nblocks * 64 * 4): one CTA per (block, group, slot); block 256 (8 warps); dynamic shared memory ldt * 4 bytes.
 __global__ void __launch_bounds__(256) lbs_table_kernel(const uint16_t *__restrict__ Wt, long ldt,
                                                         const double *__restrict__ score,
                                                         const int32_t *__restrict__ theta0, int C, int lbs_block,
                                                         double *__restrict__ table, double *__restrict__ base) {
-    const int b = blockIdx.x / kLbsGroups, g = blockIdx.x % kLbsGroups;
+    extern __shared__ uint32_t s_pk[];
+    __shared__ unsigned long long s_B[4];
+    const int slot = blockIdx.x & 3;
+    const int g = (blockIdx.x >> 2) % kLbsGroups, b = (blockIdx.x >> 2) / kLbsGroups;
     const int p0 = b * lbs_block;
     const int m = min(lbs_block, C - p0);
     if (g * 4 >= m) return;
@@ -325,32 +436,39 @@ __global__ void __launch_bounds__(256) lbs_table_kernel(const uint16_t *__restri
     int grp[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) grp[k] = theta0[p0 + g * 4 + k];
-    double *tb = table + ((long)b * kLbsGroups + g) * 4 * kLbsMax;
-    for (int e = warp; e < 4 * m; e += 8) {
-        const int slot = e / m, x = e % m;
-        double v = 0.0;
-        if (x / 4 != g) {
-            int ch[4] = {grp[0], grp[1], grp[2], grp[3]};
-            ch[slot] = theta0[p0 + x];
-            v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
-        }
-        if (lane == 0) tb[slot * kLbsMax + x] = v;
+    if (threadIdx.x < 4) s_B[threadIdx.x] = 0;
+    __syncthreads();
+    lbs_slot_prepare(Wt, ldt, score, grp, slot, s_pk, s_B);
+    __syncthreads();
+    double sc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) sc[k] = score[grp[k]];
+    double *tb = table + (((long)b * kLbsGroups + g) * 4 + slot) * kLbsMax;
+    for (int x = warp; x < m; x += 8) {
+        const int cx = theta0[p0 + x];
+        const double v = lbs_slot_candidate(Wt, ldt, sc, slot, cx, score[cx], s_pk, s_B);
+        if (lane == 0) tb[x] = v;
     }
-    if (warp == 0) {
+    if (slot == 0 && warp == 0) {
         double v = group_value_warp(Wt, ldt, score, grp[0], grp[1], grp[2], grp[3]);
         if (lane == 0) base[p0 / 4 + g] = v;
     }
 }
 
-// One CTA per block of positions: repeat { best cross-group swap by table lookup; apply if gain > 0;
-// refresh the two touched groups }.  grid (nblocks), block 512.
+// One cluster of 8 CTAs per block of positions: repeat { best cross-group swap by table lookup; apply if gain > 0;
+// refresh the two touched groups }.  Every CTA takes the same decision from the same table (no exchange needed), then
+// refreshes one of the 2 groups x 4 slots of table rows; a cluster barrier publishes the rows before the next
+// decision.  grid (nblocks * 8), cluster (8), block 512, dynamic shared memory ldt * 4 bytes.
+constexpr int kLbsCluster = 8;
 __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restrict__ Wt, long ldt,
                                                           const double *__restrict__ score,
                                                           const int32_t *__restrict__ theta0, int C, int lbs_block,
                                                           int max_swaps, double *__restrict__ table,
                                                           double *__restrict__ base, int32_t *__restrict__ theta,
                                                           unsigned long long *__restrict__ counters) {
-    const int b = blockIdx.x;
+    extern __shared__ uint32_t s_pk[];
+    const int b = blockIdx.x / kLbsCluster;
+    const int unit = blockIdx.x % kLbsCluster;                  // rank in the cluster: which (group, slot) this CTA refreshes
     const int p0 = b * lbs_block;
     const int m = min(lbs_block, C - p0);
     const int G = m / 4;
@@ -361,6 +479,7 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
     __shared__ double red_gain[16];
     __shared__ int red_idx[16];
     __shared__ int decision;      // linear pair index i*256+j, or -1 to stop
+    __shared__ unsigned long long s_B[4];
     double *tb = table + (long)b * kLbsGroups * 4 * kLbsMax;
     if (tid < m) { pos2x[tid] = tid; chan[tid] = theta0[p0 + tid]; }
     if (tid < G) s_base[tid] = base[p0 / 4 + tid];
@@ -374,7 +493,8 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
                 const int i = e >> 8, j = e & 255;
                 if (j <= i || j >= m || (i >> 2) == (j >> 2)) continue;
                 const int gi = i >> 2, si = i & 3, gj = j >> 2, sj = j & 3;
-                double after = __dadd_rn(tb[(gi * 4 + si) * kLbsMax + pos2x[j]], tb[(gj * 4 + sj) * kLbsMax + pos2x[i]]);
+                // rows of the table are rewritten by other CTAs of the cluster: read them from L2, never from this SM's L1
+                double after = __dadd_rn(__ldcg(&tb[(gi * 4 + si) * kLbsMax + pos2x[j]]), __ldcg(&tb[(gj * 4 + sj) * kLbsMax + pos2x[i]]));
                 double gain = __dsub_rn(after, __dadd_rn(s_base[gi], s_base[gj]));
                 if (gain > best || (gain == best && e < best_e)) { best = gain; best_e = e; }
             }
@@ -405,26 +525,40 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
         if (tid == 0) { int t = pos2x[bi]; pos2x[bi] = pos2x[bj]; pos2x[bj] = t; }
         ++swaps;
         __syncthreads();
-        // refresh base and table rows of the two touched groups: 2 * (1 + 4*m) group evaluations
-        const int per_group = 1 + 4 * m;
-        for (int w = warp; w < 2 * per_group; w += 16) {
-            const int g = (w < per_group) ? (bi >> 2) : (bj >> 2);
-            const int e = (w < per_group) ? w : w - per_group;
+        // refresh: this CTA's (group, slot) rows of the table; units 0 and 4 also the base value of their group
+        {
+            const int g = unit < 4 ? (bi >> 2) : (bj >> 2);
+            const int slot = unit & 3;
             int ch[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) ch[k] = chan[pos2x[g * 4 + k]];
-            if (e == 0) {
+            double sc[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sc[k] = score[ch[k]];
+            if (slot == 0 && warp == 0) {
                 double v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
-                if (lane == 0) s_base[g] = v;
-            } else {
-                const int slot = (e - 1) / m, x = (e - 1) % m;
-                ch[slot] = chan[x];
-                double v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
+                if (lane == 0) base[p0 / 4 + g] = v;
+            }
+            if (tid < 4) s_B[tid] = 0;
+            __syncthreads();
+            lbs_slot_prepare(Wt, ldt, score, ch, slot, s_pk, s_B);
+            __syncthreads();
+            for (int x = warp; x < m; x += 16) {
+                const int cx = chan[x];
+                const double v = lbs_slot_candidate(Wt, ldt, sc, slot, cx, score[cx], s_pk, s_B);
                 if (lane == 0) tb[(g * 4 + slot) * kLbsMax + x] = v;
             }
         }
+        __threadfence();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (tid < 2) {                                          // the two refreshed base values, written by units 0 and 4
+            const int g = tid == 0 ? (bi >> 2) : (bj >> 2);
+            s_base[g] = *reinterpret_cast<volatile double *>(base + p0 / 4 + g);
+        }
         __syncthreads();
     }
+    if (unit != 0) return;
     if (tid < m) theta[p0 + tid] = chan[pos2x[tid]];
     if (tid < G) base[p0 / 4 + tid] = s_base[tid];
     if (tid == 0 && swaps) atomicAdd(&counters[1], (unsigned long long)swaps);
@@ -701,11 +835,30 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     }
     if (o.use_lbs) {
         const int nblocks = ceil_div(C, o.lbs_block);
-        lbs_table_kernel<<<nblocks * kLbsGroups, 256, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, C, o.lbs_block,
-                                                                  w.table, w.base);
+        const size_t pk_smem = (size_t)w.ldt * sizeof(uint32_t);          // per-row f2 record of one (group, slot)
+        if (pk_smem > (size_t)di.max_smem_optin - 8192) return ESP_ERR_UNSUPPORTED;   // No beyond ~56000 rows
+        ESP_CUDA_OK(cudaFuncSetAttribute(lbs_table_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pk_smem));
+        ESP_CUDA_OK(cudaFuncSetAttribute(lbs_greedy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pk_smem));
+        lbs_table_kernel<<<nblocks * kLbsGroups * 4, 256, pk_smem, stream>>>(w.wt, w.ldt, w.score, w.theta0, C, o.lbs_block,
+                                                                            w.table, w.base);
         if (stats) objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective);
-        lbs_greedy_kernel<<<nblocks, 512, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, C, o.lbs_block, o.lbs_max_swaps,
-                                                        w.table, w.base, perm, w.counters);
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(nblocks * kLbsCluster);
+            cfg.blockDim = dim3(512);
+            cfg.dynamicSmemBytes = pk_smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = kLbsCluster;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, lbs_greedy_kernel, (const uint16_t *)w.wt, w.ldt, (const double *)w.score,
+                                           (const int32_t *)w.theta0, C, o.lbs_block, o.lbs_max_swaps, w.table, w.base, perm,
+                                           w.counters));
+        }
         if (stats) objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective + 1);
     } else if (stats) {
         group_values_kernel<<<ceil_div(G, 8), 256, 0, stream>>>(w.wt, w.ldt, w.score, w.theta0, G, w.base);
