@@ -474,7 +474,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--x-layout", default="channel", choices=["token", "channel"],
                     help="activation layout handed to esp_spgemm: channel = [K, M] (channels are rows)")
-    ap.add_argument("--lbs-max-swaps", type=int, default=8,
+    ap.add_argument("--lbs-max-swaps", type=int, default=0,
                     help="cap on block-shuffle swaps per block while preparing the weights (0 = run to the end)")
     ap.add_argument("--cpu-rows", type=int, default=256)
     ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "prune"],

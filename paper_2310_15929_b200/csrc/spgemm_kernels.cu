@@ -765,15 +765,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
     grid_launch_dependents();
 
     if (warp == 0) {
-        if (lane < stages) {
-            for (int it = lane + stages; it < nk; it += stages) {      // this lane's stage, every later round
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
-                if (!mbar_wait(empty(lane), ph ^ 1u, abort_flag)) break;
-                mbar_arrive_expect_tx(full(lane), kTileBytes);
-                bulk_load(sbase + lane * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(lane));
-            }
-        }
-        __syncwarp();
+        // (later weight tiles are issued by the X producer warps below, right after they have seen the stage's `empty`)
         if (split > 1) cluster_wait();
     } else if (warp == 1) {
         if (lane == 0) {
@@ -849,6 +841,13 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
                 }
             }
             cp_async_arrive_noinc(full(s));
+            // Weight tile of this stage (beyond the first `stages`, which were issued at start-up): lane 0 of producer warp
+            // s % 4.  Copies issued by one thread do not overlap and lanes spinning in one warp hold each other up, so
+            // the issuing duty rotates over the four producer warps, which have just seen `empty` anyway.
+            if (it >= prefetch && lane == 0 && (warp - 2) == (s & 3)) {
+                mbar_arrive_expect_tx(full(s), kTileBytes);
+                bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
+            }
         }
         // ---- epilogue
         const int quarter = warp & 3;
