@@ -574,7 +574,7 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
 // owned by cluster rank t % split; every CTA stores its fp32 partial rows straight into the owner's
 // shared memory (slot = sender's rank) and arrives on the owner's mbarrier; the owner adds the slots in
 // rank order -- deterministic, no global scratch, one cluster-wide rendezvous at start-up only.  (Token tiles
-// of 128 and 256, whose partial tiles would not fit beside the stages, stage them in the stage area after the
+// of 64 and more, whose partial tiles would crowd out the stages, stage them in the stage area after the
 // main loop and let each owner pull its rows from the peers instead.)
 // grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192:
 //   warp 0 lane 0  weight-tile producer        warp 1  tensor-memory allocation; lane 0: tcgen05.cp + sparse MMAs
@@ -662,10 +662,14 @@ struct StreamCfg {
     static constexpr int kStage = kTileBytes + kXStage;              // a multiple of 1024
     static constexpr uint32_t kLayout = BN >= 64 ? 2u : BN == 32 ? 4u : 6u;   // 128 / 64 / 32-byte swizzle
     static constexpr int kSwzShift = BN >= 64 ? 0 : BN == 32 ? 1 : 2;         // row bits that feed the XOR
-    static constexpr bool kPush = BN <= 64;                          // K-slice reduction by pushing (else by pulling)
+    static constexpr bool kPush = BN <= 32;                          // K-slice reduction by pushing (else by pulling)
+    // 16-byte asynchronous row copies deliver 25 / 44 / 60 GB/s per SM from 128 / 256 / 512 threads: wide X tiles get
+    // sixteen producer warps, narrow ones (little X per weight tile) four
+    static constexpr int kProd = BN >= 64 ? 512 : 128;
+    static constexpr int kThreads = 64 + kProd;
     static constexpr int kRecvBytes = kPush ? (BN + 8) * 512 : 0;    // pushed partials: [sender][128 features][rows per owner] fp32
 };
-inline size_t stream_recv_bytes(int bn, int split) { return (split > 1 && bn <= 64) ? (size_t)(bn + 8) * 512 : 0; }
+inline size_t stream_recv_bytes(int bn, int split) { return (split > 1 && bn <= 32) ? (size_t)(bn + 8) * 512 : 0; }
 inline size_t stream_smem_bytes(int bn, int stages, int split) {
     return (size_t)stages * (kTileBytes + 256 * bn) + stream_recv_bytes(bn, split) + kPermRing * 512 + 512 + 1024;
 }
@@ -693,7 +697,7 @@ __device__ __forceinline__ void push_columns_pow2(const uint32_t (&v)[16], int c
 }
 
 template <int BN>
-__global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, const int stages) {
+__global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(const GemmParams p, const int stages) {
     using L = StreamCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -724,7 +728,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
     const int cnt = (BN + split - 1) / split;                        // rows per owner (pitch of a feature's run in a slot)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(full(s), 128 + 1); mbar_init(empty(s), 1); }
+        for (int s = 0; s < stages; ++s) { mbar_init(full(s), L::kProd + 1); mbar_init(empty(s), 1); }
         mbar_init(accum_bar, 1);
         mbar_init(recv_bar, 1);
         *abort_flag = 0;
@@ -745,7 +749,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
         // permutation entries of the first stages, all loads in flight together (the X addresses depend on them)
         const int g = threadIdx.x - 64;
         int pre[kPermRing];
@@ -798,7 +802,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
         // ---- X producers: thread g copies the 16-byte pieces e = g, g + 128, ... of the stage's 128 rows
         const int g = threadIdx.x - 64;
         constexpr int kPieces = 128 * L::kChunks;                     // per token block
-        constexpr int kPerThread = (kPieces + 127) / 128;
+        constexpr int kPerThread = (kPieces + L::kProd - 1) / L::kProd;
         const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
         const bool ring_refill = nk > kPermRing;                      // long K-slices: keep the ring kPermRing stages ahead
         bool alive = true;
@@ -808,19 +812,19 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
             const int s = it % stages;
             const uint32_t ph = (uint32_t)(it / stages) & 1u;
             const int *pr = perm_s + (it % kPermRing) * 128;
-            if (ring_refill && it > 0) perm_s[((it - 1) % kPermRing) * 128 + g] = refill;   // entries of stage it-1+kPermRing
+            if (ring_refill && it > 0 && g < 128) perm_s[((it - 1) % kPermRing) * 128 + g] = refill;   // entries of stage it-1+kPermRing
             int ch[kPerThread];
 #pragma unroll
             for (int i = 0; i < kPerThread; ++i) {
-                const int e = g + 128 * i;
+                const int e = g + L::kProd * i;
                 ch[i] = (e < kPieces) ? pr[e / L::kChunks] : -1;
             }
             if (ring_refill) {
-                asm volatile("bar.sync 1, 128;" ::: "memory");       // everyone has read this stage's entries
+                asm volatile("bar.sync 1, %0;" ::"n"(L::kProd) : "memory");   // everyone has read this stage's entries
                 const int kpos = (kt_begin + it + kPermRing) * kTileK + g;
-                refill = (it + kPermRing < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
+                refill = (g < 128 && it + kPermRing < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
             }
-            // (a thread whose wait gave up keeps looping without copying: the named barrier above needs all 128)
+            // (a thread whose wait gave up keeps looping without copying: the named barrier above needs every producer)
             if (alive && !mbar_wait(empty(s), ph ^ 1u, abort_flag)) alive = false;
             if (!alive) continue;
             const uint32_t xs = sbase + s * L::kStage + kTileBytes;
@@ -828,7 +832,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
             for (int tb = 0; tb < L::kTokBlocks; ++tb) {
 #pragma unroll
                 for (int i = 0; i < kPerThread; ++i) {
-                    const int e = g + 128 * i;
+                    const int e = g + L::kProd * i;
                     if (e < kPieces) {
                         const int r = e / L::kChunks, cc = e % L::kChunks;
                         const int t = tok0 + tb * 64 + cc * 8;
@@ -844,12 +848,15 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
             // Weight tile of this stage (beyond the first `stages`, which were issued at start-up): lane 0 of producer warp
             // s % 4.  Copies issued by one thread do not overlap and lanes spinning in one warp hold each other up, so
             // the issuing duty rotates over the four producer warps, which have just seen `empty` anyway.
-            if (it >= prefetch && lane == 0 && (warp - 2) == (s & 3)) {
+            if (it >= prefetch && lane == 0 && (warp - 2) == (s & 3)) {   // (one of the first four producer warps)
                 mbar_arrive_expect_tx(full(s), kTileBytes);
                 bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
             }
         }
-        // ---- epilogue
+        // ---- epilogue: the first four producer warps, one quarter of the accumulator lanes each
+        if (warp >= 6) {
+            if (split > 1) cluster_wait();
+        } else {
         const int quarter = warp & 3;
         const int f_local = quarter * 32 + lane;
         const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
@@ -875,7 +882,7 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
                 }
             }
             tc_fence_before();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 2, 128;" ::: "memory");
             const int row_bytes = 128 * esize;
             const int chunks_per_row = row_bytes / 16;
             const int f_valid = min(128, p.N - ft * 128);
@@ -958,12 +965,13 @@ __global__ void __launch_bounds__(192) spgemm_stream_kernel(const GemmParams p, 
                 else reinterpret_cast<__half *>(p.Y)[o] = __float2half_rn(acc);
             }
         }
+        }
     }
     if (!L::kPush && split > 1) {
         cluster_sync_all();                                          // every partial tile is staged
         const bool fine = (*abort_flag == 0);
         const int f_valid = min(128, p.N - ft * 128);
-        for (int q = threadIdx.x; q < BN * 32; q += 192) {            // 4 consecutive features of one row per thread
+        for (int q = threadIdx.x; q < BN * 32; q += L::kThreads) {            // 4 consecutive features of one row per thread
             const int row = q >> 5, f0 = (q & 31) * 4;
             if ((row % split) != (int)rank) continue;
             const int t = tok0 + row;
@@ -1002,7 +1010,7 @@ esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int sp
     ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(f_tiles, t_tiles, split);
-    cfg.blockDim = dim3(192);
+    cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -1026,7 +1034,7 @@ int stream_cluster_capacity(int split, int stages) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1, 1, split);
-    cfg.blockDim = dim3(192);
+    cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
     cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
