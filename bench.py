@@ -362,6 +362,33 @@ def run_ours(args):
                            "roofline": {"bound": "hbm", "achieved": dgbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                         "frac": dgbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES,
                                         "frac_of_nominal_8TBs": dgbs / 8000.0, "of": peaks["source"]}}
+        # ---------------- decode with the layer's same-input linears pruned as one weight ----------------
+        # q,k,v (and gate,up) read the same X; pruned as one concatenated weight they share one permutation and run as one
+        # launch (the paper's Table 5 times Q/K/V that way).  Random kept values with legal metadata: timing only.
+        def random_packed(N, K):
+            vals_r = (torch.randn(N, K // 2, device=dev) * 0.02).half()
+            meta_r = torch.full((N, K // 8), 0xE4, dtype=torch.uint8, device=dev)
+            pk = torch.empty(b.esp_packed_bytes(N, K), dtype=torch.uint8, device=dev)
+            b.esp_pack(vals_r, meta_r, N, K, pk)
+            return pk
+        hidden, ffn = wl.linears["q"][0], wl.linears["gate"][0]
+        fused = [(3 * hidden, hidden), (hidden, hidden), (2 * ffn, hidden), (hidden, ffn)]
+        fpk = [random_packed(N, K) for N, K in fused]
+        fperm = [torch.randperm(K, device=dev).int() for _, K in fused]
+        fx = [torch.randn(K, DECODE_M, device=dev).half() for _, K in fused]
+        fy = [torch.empty(DECODE_M, N, dtype=torch.float16, device=dev) for N, _ in fused]
+        fo = b.esp_gemm_opts_default()
+        fo.x_layout = b.ESP_X_CHANNEL_MAJOR
+        fo.static_weights = 1
+
+        def fused_step():
+            for pk, pm, X, Y in zip(fpk, fperm, fx, fy):
+                b.esp_spgemm(X, pk, pm, Y, fo)
+        fms = graph_time(fused_step, 20)
+        fbytes = sum(gemm_bytes(DECODE_M, N, K) for N, K in fused)
+        extra["decode_fused_qkv_gateup"] = {"launches_per_layer": 4, "ms_per_step": fms, "value": fbytes / (fms * 1e-3) / 1e9,
+                                            "unit": "GB/s", "frac_of_measured_hbm": fbytes / (fms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del fpk, fx, fy
         # ---------------- dense cuBLAS fp16 on the same shapes (library call, context) ----------------
         def dense_step(xs_):
             for lin, X in zip(layer, xs_):
