@@ -228,6 +228,15 @@ esp_status_t esp_spgemm_static(const void *X, int M, int K, long ldx,
                                void *Y, long ldy, int out_dtype, void *cuda_stream);
 
 /*
+ * Exercises the failure path of the kernels' bounded waits without faulting anything (no counterpart in the paper;
+ * every barrier wait of the GEMM kernels is bounded so that a lost signal ends in a status code, not a hang): launches one
+ * tiny kernel whose wait can never be satisfied; after about a millisecond it gives up, records ESP_ERR_TIMEOUT in the
+ * device status word and returns normally.  The next esp_last_device_status() returns ESP_ERR_TIMEOUT, and the
+ * context stays usable.
+ */
+esp_status_t esp_selftest_wait_timeout(void *cuda_stream);
+
+/*
  * Reads and clears the device-side status word of the current device (synchronises the device).
  * Kernels bound every wait on a barrier; a wait that gives up records ESP_ERR_TIMEOUT here and the
  * kernel exits cleanly.  Returns ESP_OK if no kernel reported anything.

@@ -52,7 +52,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_gemm_opts_default",
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
-           "esp_spgemm_static", "esp_spgemm_plan")
+           "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -77,6 +77,8 @@ _lib.esp_spgemm.restype = c_int
 _lib.esp_spgemm.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
                             POINTER(esp_gemm_opts), c_void_p, c_size_t, c_void_p]
 _lib.esp_last_device_status.restype = c_int
+_lib.esp_selftest_wait_timeout.restype = c_int
+_lib.esp_selftest_wait_timeout.argtypes = [c_void_p]
 _lib.esp_spgemm_plan.restype = c_int
 _lib.esp_spgemm_plan.argtypes = [c_int, c_int, c_int, POINTER(esp_gemm_opts), c_int, POINTER(c_int), POINTER(c_int),
                                  POINTER(c_int), POINTER(c_int)]
@@ -217,6 +219,13 @@ def esp_spgemm_static(X, packed, perm, Y, stream=None):
     st = esp_spgemm_static_raw(X, M, K, X.stride(0), packed, perm, N, Y, Y.stride(0), out, _stream(stream))
     if st != ESP_OK:
         raise EsparseError(st, "esp_spgemm_static", "esp_spgemm_plan")
+
+
+def esp_selftest_wait_timeout(stream=None) -> None:
+    """Launches the kernel whose bounded wait runs out (see include/esparse.h); check esp_last_device_status() after."""
+    st = int(_lib.esp_selftest_wait_timeout(_stream(stream)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_selftest_wait_timeout")
 
 
 def esp_last_device_status() -> int:

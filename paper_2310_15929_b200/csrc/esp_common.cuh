@@ -73,6 +73,7 @@ struct GemmPlan {
 };
 esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan);
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o);
+esp_status_t launch_wait_timeout_selftest(cudaStream_t stream);
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm,
                            int N, void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan,
                            void *workspace, size_t workspace_bytes, cudaStream_t stream);

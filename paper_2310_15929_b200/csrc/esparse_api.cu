@@ -200,6 +200,13 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packe
                          workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
+esp_status_t esp_selftest_wait_timeout(void *cuda_stream) {
+    DeviceInfo di;
+    esp_status_t st = device_info(&di);
+    if (st != ESP_OK) return st;
+    return launch_wait_timeout_selftest((cudaStream_t)cuda_stream);
+}
+
 esp_status_t esp_last_device_status(void) {
     int h = 0, zero = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return ESP_ERR_CUDA;

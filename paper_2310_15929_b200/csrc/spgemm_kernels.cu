@@ -1118,7 +1118,34 @@ __global__ void __launch_bounds__(256) transpose_x_kernel(const uint16_t *__rest
     }
 }
 
+// A wait nobody ends: one thread polls a barrier that receives no arrival, gives up after a short limit, records
+// ESP_ERR_TIMEOUT and returns -- the same path every bounded wait of the GEMM kernels takes when it runs out.
+__global__ void wait_timeout_selftest_kernel() {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_barrier_init();
+        bool done = false;
+        for (uint32_t i = 0; i < (1u << 12) && !done; ++i) {
+            done = mbar_try_wait(smem_u32(&bar), 0);
+            if (!done) __nanosleep(64);
+        }
+        if (!done) {
+            abort_flag = 1;
+            atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
+        }
+    }
+}
+
 }  // namespace
+
+esp_status_t launch_wait_timeout_selftest(cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>();
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
 
 static long transposed_ld(int M) { return (long)((M + 15) / 16 * 16); }
 

@@ -174,6 +174,22 @@ def test_chain_of_dependent_launches_with_static_weights():
         check(acts[i + 1].cpu().numpy(), orc.product(acts[i].cpu().numpy(), vals, meta, theta))
 
 
+def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_survives():
+    """Failure detection without a fault: a wait that nothing ends gives up, the host reads ESP_ERR_TIMEOUT, the status
+    word is cleared by the read, and the next product is correct."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu, spgemm
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    b.esp_selftest_wait_timeout()
+    assert b.esp_last_device_status() == b.ESP_ERR_TIMEOUT
+    assert b.esp_last_device_status() == b.ESP_OK
+    vals, meta, theta = pruned(21, 256, 512)
+    X = np.random.default_rng(2).standard_normal((16, 512)).astype(np.float16)
+    check(spgemm(X, pack_on_gpu(vals, meta), theta, 256), orc.product(X, vals, meta, theta))
+
+
 def test_llama7b_shapes_sampled_outputs():
     """Full-size config-1 GEMM shapes in the launch configuration the benchmark times; the oracle checks a
     seeded sample of whole token rows x feature columns plus tile-boundary rows and columns."""
