@@ -383,8 +383,8 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
                                      double sx, const uint32_t *__restrict__ pk, const unsigned long long *s_B) {
     const int lane = threadIdx.x & 31;
     long long Ax = 0, D[4] = {0, 0, 0, 0};
-    for (long j = lane * 8; j < ldt; j += 256) {
-        const uint4 vx = *reinterpret_cast<const uint4 *>(Wt + (long)cx * ldt + j);
+    const uint16_t *col = Wt + (long)cx * ldt;
+    auto rows8 = [&](const uint4 &vx, long j) {
         const uint4 p0 = *reinterpret_cast<const uint4 *>(pk + j);
         const uint4 p1 = *reinterpret_cast<const uint4 *>(pk + j + 4);
         const uint32_t pkv[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
@@ -402,7 +402,17 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
 #pragma unroll
             for (int q = 0; q < 4; ++q) D[q] += (q == f2) ? wf : 0;
         }
+    };
+    // the column comes from L2: four 16-byte loads per lane are in flight before the first is used
+    long j = lane * 8;
+    for (; j + 3 * 256 < ldt; j += 4 * 256) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldg(reinterpret_cast<const uint4 *>(col + j + u * 256));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) rows8(v[u], j + u * 256);
     }
+    for (; j < ldt; j += 256) rows8(__ldg(reinterpret_cast<const uint4 *>(col + j)), j);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         Ax += __shfl_xor_sync(0xFFFFFFFFu, Ax, off);
