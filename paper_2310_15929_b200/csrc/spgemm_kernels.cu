@@ -1298,11 +1298,11 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
         const bool dependent = o.static_weights != 0;
         if (plan.kernel == ESP_KERNEL_PAIR) {
             switch (plan.token_tile) {
-                case 128: return launch_pair<2, 128>(p, stream);
-                case 192: return launch_pair<2, 192>(p, stream);
-                case 224: return launch_pair<2, 224>(p, stream);
-                case 240: return launch_pair<2, 240>(p, stream);
-                case 256: return launch_pair<1, 256>(p, stream);
+                case 128: return launch_pair<2, 128>(p, dependent, stream);
+                case 192: return launch_pair<2, 192>(p, dependent, stream);
+                case 224: return launch_pair<2, 224>(p, dependent, stream);
+                case 240: return launch_pair<2, 240>(p, dependent, stream);
+                case 256: return launch_pair<1, 256>(p, dependent, stream);
                 default: return ESP_ERR_INVALID_ARG;
             }
         }

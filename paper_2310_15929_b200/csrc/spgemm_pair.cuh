@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     cluster_sync_all();                      // both CTAs have their barriers and tensor memory before any cross-CTA signal
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    grid_launch_dependents();                // (static_weights) the next launch may be set up while this one runs
 
     if (warp == 0) {
         // idle: keeps the producer warps at indices 2..17 (tensor-memory lane quarter = warp index % 4)
@@ -230,6 +231,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         int nxt[kAhead][2];
 #pragma unroll
         for (int u = 0; u < kAhead; ++u) { nxt[u][0] = channel_of(u, rg); nxt[u][1] = channel_of(u, rg + 64); }
+        grid_dependency_wait();              // (static_weights) X and Y may belong to the preceding kernel until it is done
         for (int it0 = 0; it0 < nk; it0 += kAhead) {
 #pragma unroll
             for (int u = 0; u < kAhead; ++u) {
@@ -351,7 +353,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 }
 
 template <int NA, int TN>
-esp_status_t launch_pair(const GemmParams &p, cudaStream_t stream) {
+esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream) {
     using L = PairCfg<NA, TN>;
     auto kern = spgemm_pair_kernel<NA, TN>;
     ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
@@ -361,13 +363,15 @@ esp_status_t launch_pair(const GemmParams &p, cudaStream_t stream) {
     cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = L::kTotal;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = dependent ? 2 : 1;
     ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
     return ESP_OK;
 }
