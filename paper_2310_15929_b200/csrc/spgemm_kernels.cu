@@ -13,6 +13,8 @@
 
 #include <cuda.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 
@@ -1045,7 +1047,26 @@ int stream_cluster_capacity(int split, int stages) {
     cfg.numAttrs = 1;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
-    return n;
+    // The occupancy calculator answers with one CTA per SM for these kernels whatever their size (it cannot know how much
+    // tensor memory a CTA will allocate); CTAs do share an SM when shared memory, threads and tensor-memory columns
+    // allow.  So its answer is taken as the packing of clusters onto GPCs at the calculator's CTAs per SM and scaled.
+    int api_per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_per_sm, kern, StreamCfg<BN>::kThreads, smem) != cudaSuccess || api_per_sm < 1) {
+        cudaGetLastError();
+        api_per_sm = 1;
+    }
+    int dev = 0, smem_per_sm = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    int per_sm = (int)((size_t)smem_per_sm / (smem + 1024));
+    per_sm = per_sm < 2048 / StreamCfg<BN>::kThreads ? per_sm : 2048 / StreamCfg<BN>::kThreads;
+    per_sm = per_sm < 512 / (int)tmem_cols_for(BN) ? per_sm : 512 / (int)tmem_cols_for(BN);
+    if (per_sm < api_per_sm) per_sm = api_per_sm;
+    const int clusters = (int)((long)n * per_sm / api_per_sm);
+    if (getenv("ESP_LOG"))
+        fprintf(stderr, "esparse occupancy tile=%d split=%d stages=%d smem=%zu: calculator clusters=%d at %d CTAs/SM, taken %d at %d CTAs/SM\n", BN,
+                split, stages, smem, n, api_per_sm, clusters, per_sm);
+    return clusters;
 }
 
 #include "spgemm_pair.cuh"
@@ -1245,9 +1266,14 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
                 if (cap <= 0) continue;
                 const long ctas = tiles * split;
                 const long waves = (ctas + cap - 1) / cap;
-                double cost = (double)waves * (kts + 2.0) + (split > 1 ? 0.25 + 0.05 * split : 0.0) + 0.01 * r;
+                // (2, 4 or 8 slices push their partial rows as vectors; other counts go element by element: measured ~2 us slower)
+                const bool pow2 = (split & (split - 1)) == 0;
+                double cost = (double)waves * (kts + 2.0) + (split > 1 ? (pow2 ? 0.25 : 6.0) + 0.05 * split : 0.0) + 0.01 * r;
                 // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
                 if (o.static_weights && 2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin) cost += 3.0;
+                if (getenv("ESP_LOG"))
+                    fprintf(stderr, "esparse plan M=%d N=%d K=%d tile=%d: split=%d stages=%d capacity=%d ctas=%ld waves=%ld cost=%.2f\n", M, N, K,
+                            bn, split, stages, cap, ctas, waves, cost);
                 if (cost < best_cost) { best_cost = cost; best_split = split; best_stages = stages; }
             }
         }
