@@ -58,7 +58,10 @@ typedef struct {
     size_t struct_size;          /* = sizeof(esp_prune_opts)                                         */
     double alpha;                /* weight of the norm in Eq. 3; the paper gives no value             */
     int bins;                    /* K of Eq. 1 (paper: 100); 2..1024                                  */
-    int n_keep, m_group;         /* N:M pattern; only 2:4 is implemented on the GPU                   */
+    int n_keep, m_group;         /* N:M pattern: 2:4, or 4:8 (Table 1's second pattern: metric, global shuffle,
+                                    selection and compression only -- use_lbs must be 0 and packed NULL,
+                                    no tensor-core form exists; meta then holds one byte per group of 8,
+                                    bit p = position p kept, vals the 4 kept weights in position order)   */
     int lbs_block;               /* m of the local block shuffle (paper: 256); multiple of 4, <= 256  */
     int lbs_max_swaps;           /* cap on swaps per block; 0 = until no swap improves (Algorithm 1)  */
     int use_entropy;             /* 0 drops IR_c from the score (norm-only baseline of Table 4)       */

@@ -270,6 +270,32 @@ def select_compress(W: np.ndarray, s: np.ndarray, theta: np.ndarray):
     return vals.reshape(No, C // 2), meta, near
 
 
+def select_compress_nm(W: np.ndarray, s: np.ndarray, theta: np.ndarray, n_keep: int = 4, m_group: int = 8):
+    """General N:M selection (the paper's 4:8 rows of Table 1; "prune N values out of M consecutive values in the
+    channel dimension"): per row and per group of M consecutive permuted channels keep the n_keep largest xi (ties: lower
+    position first).  There is no tensor-core form for 4:8, so the compressed form is plain: vals[j, g*n_keep + e] =
+    the kept weights of group g in position order (bit copies), mask[j, g*M/8 + b] = bit p%8 set iff position p = 8b + p%8
+    of the group is kept.  Returns (vals f16 [No, C*n_keep/M], mask u8 [No, C/8], near_tie bool [No, C/M]) where a
+    near-tie is a relative gap < 1e-6 between the last kept and the first dropped metric."""
+    W = np.asarray(W, dtype=np.float16)
+    No, C = W.shape
+    assert m_group % 8 == 0 and C % m_group == 0 and 0 < n_keep < m_group
+    G = C // m_group
+    theta = np.asarray(theta, dtype=np.int64)
+    Wp = W[:, theta]
+    xi = (np.abs(Wp.astype(np.float64)) * np.asarray(s, dtype=np.float64)[theta][None, :]).reshape(No, G, m_group)
+    rank = np.argsort(-xi, axis=2, kind="stable")
+    keep = np.sort(rank[:, :, :n_keep], axis=2)
+    Wg = Wp.reshape(No, G, m_group)
+    vals = np.take_along_axis(Wg, keep, axis=2)
+    kept = np.zeros((No, G, m_group), dtype=bool)
+    np.put_along_axis(kept, keep, True, axis=2)
+    mask = np.packbits(kept.reshape(No, C), axis=1, bitorder="little")
+    xs = np.take_along_axis(xi, rank, axis=2)
+    near = (xs[:, :, n_keep - 1] - xs[:, :, n_keep]) < NEAR_TIE_REL * xs[:, :, n_keep - 1]
+    return vals.reshape(No, G * n_keep), mask, near
+
+
 def unpack_meta(meta: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     """meta u8 [No, C/8] -> (idx0, idx1) int arrays [No, C/4]."""
     meta = np.asarray(meta, dtype=np.uint8)

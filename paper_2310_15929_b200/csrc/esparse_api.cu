@@ -29,7 +29,9 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 static esp_status_t check_prune_opts(const esp_prune_opts *o) {
     if (!o || o->struct_size != sizeof(esp_prune_opts)) return ESP_ERR_INVALID_ARG;
-    if (o->n_keep != 2 || o->m_group != 4) return ESP_ERR_UNSUPPORTED;
+    const bool is24 = (o->n_keep == 2 && o->m_group == 4), is48 = (o->n_keep == 4 && o->m_group == 8);
+    if (!is24 && !is48) return ESP_ERR_UNSUPPORTED;
+    if (is48 && o->use_lbs) return ESP_ERR_UNSUPPORTED;      // 4:8: metric, global shuffle, selection, compression only
     if (o->bins < 2 || o->bins > 512) return ESP_ERR_UNSUPPORTED;
     if (o->lbs_block < 4 || o->lbs_block > 256 || o->lbs_block % 4 != 0) return ESP_ERR_INVALID_ARG;
     if (o->lbs_max_swaps < 0) return ESP_ERR_INVALID_ARG;
@@ -117,6 +119,7 @@ esp_status_t esp_metric_prune(const void *W, int No, int C, long ldw, const void
     esp_status_t st = check_prune_opts(opts);
     if (st != ESP_OK) return st;
     if (!W || !vals || !meta || !perm) return ESP_ERR_INVALID_ARG;
+    if (opts->m_group == 8 && packed) return ESP_ERR_UNSUPPORTED;    // no tensor-core form of 4:8: nothing to pack
     if (!Xcal && !opts->score_override) return ESP_ERR_INVALID_ARG;
     if (stats && stats->struct_size != sizeof(esp_prune_stats)) return ESP_ERR_INVALID_ARG;
     if (No <= 0 || C <= 0 || C % 8 != 0 || ldw < C) return ESP_ERR_SHAPE;

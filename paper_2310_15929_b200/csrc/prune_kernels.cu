@@ -213,7 +213,7 @@ __global__ void mean_metric_kernel(int C, int No, const unsigned long long *__re
 // mean metric; the channel of rank r goes to group r mod G, slot r div G (neighbours in rank never share
 // a group).
 // --------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__restrict__ mean, int use_gns,
+__global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__restrict__ mean, int use_gns, int m_group,
                                                        int32_t *__restrict__ theta0) {
     __shared__ double tile[256];
     const int c = blockIdx.x * 256 + threadIdx.x;
@@ -234,8 +234,8 @@ __global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__re
         }
     }
     if (c < C) {
-        const int G = C / 4;
-        theta0[(rank % G) * 4 + rank / G] = c;
+        const int G = C / m_group;
+        theta0[(rank % G) * m_group + rank / G] = c;
     }
 }
 
@@ -653,6 +653,64 @@ __global__ void __launch_bounds__(256) select_compress_kernel(const __half *__re
     if ((threadIdx.x & 31) == 0 && near) atomicAdd(&counters[0], (unsigned long long)near);
 }
 
+// 4-of-8 selection + compression (the 4:8 pattern of the paper's Table 1; no tensor-core form exists for it, so the
+// output is plain: 4 kept values per group in position order and one mask byte per group, bit p = position p kept).
+// One CTA per output row, one thread per group of 8 permuted positions.
+__global__ void __launch_bounds__(256) select_compress_48_kernel(const __half *__restrict__ W, int No, int C, long ldw,
+                                                                 const double *__restrict__ score,
+                                                                 const int32_t *__restrict__ theta,
+                                                                 __half *__restrict__ vals, uint8_t *__restrict__ mask,
+                                                                 unsigned long long *__restrict__ counters) {
+    extern __shared__ uint16_t s_row[];
+    const int j = blockIdx.x;
+    const uint16_t *Wr = reinterpret_cast<const uint16_t *>(W) + (long)j * ldw;
+    for (int c = threadIdx.x * 8; c < C; c += 256 * 8)
+        *reinterpret_cast<uint4 *>(s_row + c) = __ldg(reinterpret_cast<const uint4 *>(Wr + c));
+    __syncthreads();
+    unsigned int near = 0;
+    for (int u = threadIdx.x; u < C / 8; u += 256) {
+        uint16_t h[8];
+        double xi[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int c = theta[u * 8 + k];
+            h[k] = s_row[c];
+            xi[k] = __dmul_rn(half_bits_abs_to_double(h[k]), score[c]);
+        }
+        uint16_t out[4] = {0, 0, 0, 0};
+        unsigned int byte = 0;
+        int nk = 0;
+        double fourth = 0.0, fifth = 0.0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            int ahead = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (q == k) continue;
+                ahead += (xi[q] > xi[k] || (xi[q] == xi[k] && q < k)) ? 1 : 0;
+            }
+            if (ahead < 4) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (e == nk) out[e] = h[k];
+                ++nk;
+                byte |= 1u << k;
+            }
+            if (ahead == 3) fourth = xi[k];
+            if (ahead == 4) fifth = xi[k];
+        }
+        if (__dsub_rn(fourth, fifth) < __dmul_rn(1e-6, fourth)) ++near;
+        uint2 packed;
+        packed.x = (unsigned int)out[0] | ((unsigned int)out[1] << 16);
+        packed.y = (unsigned int)out[2] | ((unsigned int)out[3] << 16);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(vals) + (long)j * (C / 2) + u * 4) = packed;
+        mask[(long)j * (C / 8) + u] = (uint8_t)byte;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) near += __shfl_xor_sync(0xFFFFFFFFu, near, off);
+    if ((threadIdx.x & 31) == 0 && near) atomicAdd(&counters[0], (unsigned long long)near);
+}
+
 // --------------------------------------------------------------------------------------------------
 // K7: re-tile (vals, meta) into the layout the sparse MMA reads.
 // Per (feature tile ft, channel tile kt) 18432 contiguous bytes:
@@ -835,7 +893,7 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     if (o.perm_override)
         ESP_CUDA_OK(cudaMemcpyAsync(theta0, o.perm_override, sizeof(int32_t) * C, cudaMemcpyDeviceToDevice, stream));
     else
-        gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, theta0);
+        gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, o.m_group, theta0);
     ESP_CUDA_OK(cudaGetLastError());
 
     // K5
@@ -881,7 +939,11 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     // K6 + K7
     const size_t row_smem = sizeof(uint16_t) * (size_t)C;
     ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_smem));
-    select_compress_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
+    if (o.m_group == 8) {
+        ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_48_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_smem));
+        select_compress_48_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
+    } else
+        select_compress_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
     ESP_CUDA_OK(cudaGetLastError());
     if (packed) {
         st = launch_pack(vals, meta, No, C, packed, stream);

@@ -159,3 +159,32 @@ def test_decompress_and_pack_roundtrip():
     assert np.array_equal(unsw.view(np.uint16), ref.vals[:128, :64].view(np.uint16))
     nibbles = packed[:, :, 16384:]
     assert set(np.unique(nibbles & 0xF).tolist()) | set(np.unique(nibbles >> 4).tolist()) <= set(orc.LEGAL_NIBBLES)
+
+
+@pytest.mark.parametrize("No,C,T", [(96, 256, 200), (200, 1024, 130)])
+def test_four_of_eight_pattern(No, C, T):
+    """4:8 (Table 1's second pattern): statistics, score, global shuffle in groups of 8, 4-of-8 selection and compression
+    against the oracle, bit-exact; the library refuses what 4:8 has no form for."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import GpuPrune
+    W, X = layer(70 + C, No, C, T)
+    alpha = 1.0 / math.sqrt(T)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), alpha)
+    theta0, _ = orc.global_naive_shuffle(orc.channel_mean_metric(W, s), m_group=8)
+    vals_ref, mask_ref, near = orc.select_compress_nm(W, s, theta0, 4, 8)
+    gp = GpuPrune(W, X, alpha, stats=True, pack=False, n_keep=4, m_group=8, use_lbs=0)
+    vals, mask, perm = gp.host()
+    assert np.array_equal(perm, theta0)
+    bad = np.argwhere(mask != mask_ref)
+    for j, g in bad:
+        assert near[j, g], (j, g)
+    if len(bad) == 0:
+        assert np.array_equal(vals.view(np.uint16), vals_ref.view(np.uint16))
+    assert gp.stats.near_tie_groups == int(near.sum())
+    with pytest.raises(b.EsparseError) as e:
+        GpuPrune(W, X, alpha, stats=False, pack=False, n_keep=4, m_group=8, use_lbs=1)
+    assert e.value.status == b.ESP_ERR_UNSUPPORTED
+    with pytest.raises(b.EsparseError) as e:
+        GpuPrune(W, X, alpha, stats=False, pack=True, n_keep=4, m_group=8, use_lbs=0)
+    assert e.value.status == b.ESP_ERR_UNSUPPORTED

@@ -355,6 +355,49 @@ def test_select_two_of_four_legal_nibbles_bit_copies_and_bruteforce():
     assert not near.any() or near.dtype == bool
 
 
+def test_select_four_of_eight_counts_bit_copies_bruteforce_and_two_of_four_consistency():
+    """The 4:8 pattern of the paper's Table 1: exactly 4 kept per group of 8, kept values are bit copies in position
+    order, the kept set maximises the retained metric over all C(8,4) = 70 masks, and the general routine run as 2:4
+    reproduces the dedicated 2:4 routine (values and positions)."""
+    W, X = rand_layer(60, 24, 64, 90)
+    s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.3)
+    theta = np.random.default_rng(61).permutation(64).astype(np.int32)
+    vals, mask, near = orc.select_compress_nm(W, s, theta, 4, 8)
+    assert vals.shape == (24, 32) and mask.shape == (24, 8) and near.shape == (24, 8)
+    kept = np.unpackbits(mask, axis=1, bitorder="little").astype(bool)
+    assert np.all(kept.reshape(24, 8, 8).sum(axis=2) == 4)
+    Wp = W[:, theta]
+    assert np.array_equal(Wp.view(np.uint16)[kept].reshape(24, 32), vals.view(np.uint16))
+    xi = orc.metric(W, s)[:, theta].reshape(24, 8, 8)
+    for j in range(24):
+        for g in range(8):
+            best = max(sum(xi[j, g, list(c)]) for c in itertools.combinations(range(8), 4))
+            got = xi[j, g][kept[j, 8 * g:8 * g + 8]].sum()
+            assert abs(got - best) < 1e-12
+    # 2:4 through the general routine needs M % 8 == 0 for the byte mask, so compare on M = 8, N = 4 against two 2:4 groups
+    # only where both agree by construction: a group of 8 whose kept set is 2 + 2 is also what 2:4 keeps
+    v2, meta2, _ = orc.select_compress(W, s, theta)
+    i0, i1 = orc.unpack_meta(meta2)
+    kept24 = np.zeros((24, 16, 4), dtype=bool)
+    np.put_along_axis(kept24, i0[:, :, None], True, axis=2)
+    np.put_along_axis(kept24, i1[:, :, None], True, axis=2)
+    kept24 = kept24.reshape(24, 64)
+    # 4:8 keeps at least as much metric as 2:4 (every 2:4 mask is a 4:8 mask), group by group
+    xi_flat = xi.reshape(24, 64)
+    r48 = (xi_flat * kept).reshape(24, 8, 8).sum(axis=2)
+    r24 = (xi_flat * kept24).reshape(24, 8, 8).sum(axis=2)
+    assert np.all(r48 >= r24 - 1e-12) and np.any(r48 > r24 + 1e-9)
+
+
+def test_select_four_of_eight_tie_break_lower_position():
+    W = np.ones((1, 8), dtype=np.float16)
+    vals, mask, near = orc.select_compress_nm(W, np.ones(8), np.arange(8, dtype=np.int32), 4, 8)
+    assert mask[0, 0] == 0x0F and near[0, 0]
+    W[0] = [1, 2, 1, 2, 1, 2, 1, 2]
+    vals, mask, near = orc.select_compress_nm(W, np.ones(8), np.arange(8, dtype=np.int32), 4, 8)
+    assert mask[0, 0] == 0xAA and np.array_equal(vals[0], np.full(4, 2, dtype=np.float16)) and not near[0, 0]
+
+
 def test_select_tie_break_lower_position():
     W = np.array([[1, 1, 1, 1, 2, 1, 2, 1]], dtype=np.float16)
     s = np.ones(8)
