@@ -123,6 +123,28 @@ esp_status_t esp_metric_prune(const void *W, int No, int C, long ldw,
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Streaming calibration: the channel statistics of Eq. 1-3 accumulated over many chunks of activations (the paper
+ * calibrates on 128 sequences) without holding them all at once.  Per-channel bins need the channel's range first,
+ * so the chunks are passed twice:
+ *
+ *   esp_calib_reset(state)                          once
+ *   esp_calib_range(state, chunk)                   every chunk: sum of squares, minimum, maximum
+ *   esp_calib_histogram(state, chunk)               every chunk again: bin counts on the final [min, max]
+ *   esp_calib_finish(state, T_total, opts, ...)     AM_c, IR_c, s_c  ->  pass s_c as opts->score_override to
+ *                                                   esp_metric_prune (Xcal = NULL)
+ *
+ * The result equals esp_metric_prune's on the concatenated chunks: counts and ranges exactly, the norm up to the order
+ * of its fp64 additions.  `state` is esp_calib_state_bytes(C, bins) bytes of caller-owned device memory; chunks are
+ * [T, C] fp16 with leading dimension ldx; bins is opts->bins (100 in the paper) in every call.
+ */
+size_t esp_calib_state_bytes(int C, int bins);
+esp_status_t esp_calib_reset(void *state, int C, int bins, void *cuda_stream);
+esp_status_t esp_calib_range(void *state, const void *X, int T, int C, long ldx, int bins, void *cuda_stream);
+esp_status_t esp_calib_histogram(void *state, const void *X, int T, int C, long ldx, int bins, void *cuda_stream);
+esp_status_t esp_calib_finish(void *state, int C, long long T_total, const esp_prune_opts *opts, double *chan_norm,
+                              double *chan_entropy, double *chan_score, void *cuda_stream);
+
+/*
  * Re-tiles (vals, meta) as written by esp_metric_prune into the packed form (step (1) of "Efficient
  * Sparse-GEMM Implementation": the compressed format the GEMM reads).  Same shapes as above.
  */
@@ -150,8 +172,12 @@ enum { ESP_KERNEL_AUTO = 0,
                                     slowly to feed the MMA; kept for comparison)                        */
        ESP_KERNEL_STREAM = 4,    /* channel-major X rows streamed by asynchronous 16-byte copies, weight
                                     tiles by bulk copies; every token count (default up to 256 tokens)  */
-       ESP_KERNEL_PAIR = 5 };    /* large M: two SMs share one 512-feature x token_tile MMA tile
-                                    (token_tile 240 by default; 128, 192, 224 or 256 on request)        */
+       ESP_KERNEL_PAIR = 5,      /* large M: two SMs share one 512-feature x token_tile MMA tile
+                                    (token_tile 240 by default; 128, 192, 224 or 256 on request); X rows
+                                    are gathered through the permutation by 16-byte copies              */
+       ESP_KERNEL_PAIR_TILED = 6 };/* the same tile, fed by bulk copies: a pass over X first writes the
+                                    permuted, swizzled operand images into the workspace (default for
+                                    large M when the workspace has room; token_tile 128..240)           */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
@@ -171,9 +197,12 @@ typedef struct {
 void esp_gemm_opts_default(esp_gemm_opts *opts);
 
 /*
- * Bytes of device workspace esp_spgemm can use.  0 for channel-major X.  For token-major X it is the size
- * of a transposed (channels-as-rows, not permuted) copy of X, which lets the fast kernels run; with a NULL
- * or smaller workspace the call still works through the element-gather kernel.
+ * Bytes of device workspace esp_spgemm can use: for token-major X a transposed (channels-as-rows, not
+ * permuted) copy of X, which lets the fast kernels run, and for more than 256 tokens the permuted X operand
+ * images of ESP_KERNEL_PAIR_TILED (about 2.2 * M * K bytes).  With a smaller workspace the call still works:
+ * without room for the images through ESP_KERNEL_PAIR, without room for the transposed copy (or with
+ * NULL) through the element-gather kernel.  The workspace is scratch: nothing in it outlives the call's work
+ * on the stream, and calls on different streams need different workspaces.
  */
 size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts);
 

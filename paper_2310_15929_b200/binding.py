@@ -18,7 +18,7 @@ ESP_ERR_STATIC_LIMIT = 8
 ESP_STATIC_SCRATCH_BYTES = 8 << 20
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
-ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR = 0, 1, 2, 4, 5
+ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR, ESP_KERNEL_PAIR_TILED = 0, 1, 2, 4, 5, 6
 
 
 class esp_prune_opts(ctypes.Structure):
@@ -52,7 +52,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_gemm_opts_default",
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
-           "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout")
+           "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout", "esp_calib_state_bytes", "esp_calib_reset",
+           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -226,6 +227,47 @@ def esp_selftest_wait_timeout(stream=None) -> None:
     st = int(_lib.esp_selftest_wait_timeout(_stream(stream)))
     if st != ESP_OK:
         raise EsparseError(st, "esp_selftest_wait_timeout")
+
+
+_lib.esp_calib_state_bytes.restype = c_size_t
+_lib.esp_calib_state_bytes.argtypes = [c_int, c_int]
+_lib.esp_calib_reset.restype = c_int
+_lib.esp_calib_reset.argtypes = [c_void_p, c_int, c_int, c_void_p]
+_lib.esp_calib_range.restype = c_int
+_lib.esp_calib_range.argtypes = [c_void_p, c_void_p, c_int, c_int, c_long, c_int, c_void_p]
+_lib.esp_calib_histogram.restype = c_int
+_lib.esp_calib_histogram.argtypes = [c_void_p, c_void_p, c_int, c_int, c_long, c_int, c_void_p]
+_lib.esp_calib_finish.restype = c_int
+_lib.esp_calib_finish.argtypes = [c_void_p, c_int, c_longlong, POINTER(esp_prune_opts), c_void_p, c_void_p, c_void_p, c_void_p]
+
+
+def esp_calib_state_bytes(C: int, bins: int) -> int:
+    return int(_lib.esp_calib_state_bytes(C, bins))
+
+
+def _calib_call(fn, name, *args):
+    st = int(fn(*args))
+    if st != ESP_OK:
+        raise EsparseError(st, name)
+
+
+def esp_calib_reset(state, C, bins, stream=None):
+    _calib_call(_lib.esp_calib_reset, "esp_calib_reset", _ptr(state), C, bins, _stream(stream))
+
+
+def esp_calib_range(state, X, bins, stream=None):
+    _calib_call(_lib.esp_calib_range, "esp_calib_range", _ptr(state), _ptr(X), X.shape[0], X.shape[1], X.stride(0), bins,
+                _stream(stream))
+
+
+def esp_calib_histogram(state, X, bins, stream=None):
+    _calib_call(_lib.esp_calib_histogram, "esp_calib_histogram", _ptr(state), _ptr(X), X.shape[0], X.shape[1], X.stride(0),
+                bins, _stream(stream))
+
+
+def esp_calib_finish(state, C, T_total, opts, chan_norm, chan_entropy, chan_score, stream=None):
+    _calib_call(_lib.esp_calib_finish, "esp_calib_finish", _ptr(state), C, T_total, ctypes.byref(opts), _ptr(chan_norm),
+                _ptr(chan_entropy), _ptr(chan_score), _stream(stream))
 
 
 def esp_last_device_status() -> int:

@@ -64,15 +64,30 @@ esp_status_t launch_pack(const __half *vals, const uint8_t *meta, int No, int C,
 esp_status_t launch_decompress(const __half *vals, const uint8_t *meta, const int32_t *perm, int No, int C,
                                __half *out, long ldw, cudaStream_t stream);
 
+// ---- streaming calibration (prune_kernels.cu)
+struct CalibState {
+    double *sumsq, *lo, *hi, *norm;
+    unsigned int *counts;
+    double *part_sumsq; float *part_min; float *part_max;
+    size_t total_bytes;
+};
+CalibState carve_calib_state(void *state, int C, int bins);
+esp_status_t launch_calib_reset(const CalibState &c, int C, int bins, cudaStream_t stream);
+esp_status_t launch_calib_range(const CalibState &c, const __half *X, int T, int C, long ldx, cudaStream_t stream);
+esp_status_t launch_calib_histogram(const CalibState &c, const __half *X, int T, int C, long ldx, int bins, cudaStream_t stream);
+esp_status_t launch_calib_finish(const CalibState &c, int C, int bins, long long T_total, const esp_prune_opts &o, double *chan_norm,
+                                 double *chan_entropy, double *chan_score, cudaStream_t stream);
+
 // ---- GEMM launchers (spgemm_kernels.cu) ------------------------------------------------------------
 struct GemmPlan {
-    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA | ESP_KERNEL_STREAM | ESP_KERNEL_PAIR
+    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA | ESP_KERNEL_STREAM | ESP_KERNEL_PAIR | ESP_KERNEL_PAIR_TILED
     int token_tile;    // MMA N
     int split_k;       // cluster size along K
     int stages;
 };
-esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan);
-size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o);
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan);
+size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o);        // everything any plan could use
+size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o);    // below this only the gather kernel runs
 esp_status_t launch_wait_timeout_selftest(cudaStream_t stream);
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm,
                            int N, void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan,

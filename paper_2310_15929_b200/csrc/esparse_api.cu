@@ -44,7 +44,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->out_dtype != ESP_OUT_F16 && o->out_dtype != ESP_OUT_F32) return ESP_ERR_INVALID_ARG;
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
     if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
-        o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR)
+        o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR && o->force_kernel != ESP_KERNEL_PAIR_TILED)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
@@ -139,6 +139,56 @@ esp_status_t esp_metric_prune(const void *W, int No, int C, long ldw, const void
                         (cudaStream_t)cuda_stream);
 }
 
+size_t esp_calib_state_bytes(int C, int bins) {
+    if (C <= 0 || C % 8 != 0 || bins < 2 || bins > 512) return 0;
+    return carve_calib_state(nullptr, C, bins).total_bytes;
+}
+
+static esp_status_t check_calib(const void *state, int C, int bins) {
+    if (!state) return ESP_ERR_INVALID_ARG;
+    if (C <= 0 || C % 8 != 0) return ESP_ERR_SHAPE;
+    if (bins < 2 || bins > 512) return ESP_ERR_UNSUPPORTED;
+    if (!aligned16(state)) return ESP_ERR_ALIGNMENT;
+    return ESP_OK;
+}
+
+esp_status_t esp_calib_reset(void *state, int C, int bins, void *cuda_stream) {
+    esp_status_t st = check_calib(state, C, bins);
+    if (st != ESP_OK) return st;
+    return launch_calib_reset(carve_calib_state(state, C, bins), C, bins, (cudaStream_t)cuda_stream);
+}
+
+static esp_status_t check_chunk(const void *X, int T, int C, long ldx) {
+    if (!X) return ESP_ERR_INVALID_ARG;
+    if (T <= 0 || ldx < C) return ESP_ERR_SHAPE;
+    if (ldx % 8 != 0 || !aligned16(X)) return ESP_ERR_ALIGNMENT;
+    return ESP_OK;
+}
+
+esp_status_t esp_calib_range(void *state, const void *X, int T, int C, long ldx, int bins, void *cuda_stream) {
+    esp_status_t st = check_calib(state, C, bins);
+    if (st == ESP_OK) st = check_chunk(X, T, C, ldx);
+    if (st != ESP_OK) return st;
+    return launch_calib_range(carve_calib_state(state, C, bins), (const __half *)X, T, C, ldx, (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_calib_histogram(void *state, const void *X, int T, int C, long ldx, int bins, void *cuda_stream) {
+    esp_status_t st = check_calib(state, C, bins);
+    if (st == ESP_OK) st = check_chunk(X, T, C, ldx);
+    if (st != ESP_OK) return st;
+    return launch_calib_histogram(carve_calib_state(state, C, bins), (const __half *)X, T, C, ldx, bins, (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_calib_finish(void *state, int C, long long T_total, const esp_prune_opts *opts, double *chan_norm,
+                              double *chan_entropy, double *chan_score, void *cuda_stream) {
+    if (!opts || opts->struct_size != sizeof(esp_prune_opts) || !chan_score) return ESP_ERR_INVALID_ARG;
+    esp_status_t st = check_calib(state, C, opts->bins);
+    if (st != ESP_OK) return st;
+    if (T_total <= 0 || T_total > 0x7FFFFFFFLL) return ESP_ERR_SHAPE;
+    return launch_calib_finish(carve_calib_state(state, C, opts->bins), C, opts->bins, T_total, *opts, chan_norm, chan_entropy,
+                               chan_score, (cudaStream_t)cuda_stream);
+}
+
 esp_status_t esp_pack(const void *vals, const void *meta, int No, int C, void *packed, void *cuda_stream) {
     if (!vals || !meta || !packed) return ESP_ERR_INVALID_ARG;
     if (No <= 0 || C <= 0 || C % 8 != 0) return ESP_ERR_SHAPE;
@@ -172,7 +222,7 @@ esp_status_t esp_spgemm_plan(int M, int N, int K, const esp_gemm_opts *opts, int
     if (st != ESP_OK) return st;
     if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
     GemmPlan plan;
-    st = plan_gemm(M, N, K, *opts, have_workspace != 0, &plan);
+    st = plan_gemm(M, N, K, *opts, have_workspace != 0 ? gemm_workspace_bytes(M, K, *opts) : 0, &plan);
     if (st != ESP_OK) return st;
     if (kernel) *kernel = plan.kernel;
     if (token_tile) *token_tile = plan.token_tile;
@@ -196,8 +246,8 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packe
     if (st != ESP_OK) return st;
     if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
     GemmPlan plan;
-    const bool have_ws = workspace && workspace_bytes >= gemm_workspace_bytes(M, K, *opts) && aligned16(workspace);
-    st = plan_gemm(M, N, K, *opts, have_ws, &plan);
+    const bool have_ws = workspace && aligned16(workspace);
+    st = plan_gemm(M, N, K, *opts, have_ws ? workspace_bytes : 0, &plan);
     if (st != ESP_OK) return st;
     return launch_spgemm((const __half *)X, M, K, ldx, packed, perm, N, Y, ldy, *opts, plan, workspace,
                          workspace_bytes, (cudaStream_t)cuda_stream);

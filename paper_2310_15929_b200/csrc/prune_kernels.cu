@@ -93,6 +93,33 @@ __global__ void colstats_finish_kernel(int C, int splits, const double *__restri
     hi[c] = (double)mx;
 }
 
+// Streaming calibration: fold one chunk's partial statistics into the running state (chunk order = call order).
+__global__ void calib_merge_kernel(int C, int splits, const double *__restrict__ part_sumsq, const float *__restrict__ part_min,
+                                   const float *__restrict__ part_max, double *__restrict__ sumsq, double *__restrict__ lo,
+                                   double *__restrict__ hi) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double a = 0.0;
+    float mn = INFINITY, mx = -INFINITY;
+    for (int s = 0; s < splits; ++s) {
+        a = __dadd_rn(a, part_sumsq[(long)s * C + c]);
+        mn = fminf(mn, part_min[(long)s * C + c]);
+        mx = fmaxf(mx, part_max[(long)s * C + c]);
+    }
+    sumsq[c] = __dadd_rn(sumsq[c], a);
+    lo[c] = fmin(lo[c], (double)mn);
+    hi[c] = fmax(hi[c], (double)mx);
+}
+__global__ void calib_reset_kernel(int C, int bins, double *sumsq, double *lo, double *hi, unsigned int *counts) {
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < C) { sumsq[i] = 0.0; lo[i] = INFINITY; hi[i] = -INFINITY; }
+    if (i < (long)C * bins) counts[i] = 0u;
+}
+__global__ void calib_norm_kernel(int C, const double *__restrict__ sumsq, double *__restrict__ norm) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < C) norm[c] = sqrt(sumsq[c]);
+}
+
 // --------------------------------------------------------------------------------------------------
 // K2: per-channel histogram with K equal-width bins on [lo_c, hi_c] (Eq. 1's bins), exact integer counts.
 // bin = min(K-1, floor((x - lo) * K / (hi - lo))) in fp64: the numerator is exact and the quotient is
@@ -833,6 +860,65 @@ esp_status_t launch_pack(const __half *vals, const uint8_t *meta, int No, int C,
     const int k_tiles = ceil_div(C, kTileK), f_tiles = ceil_div(No, kTileFeat);
     pack_kernel<<<dim3(k_tiles, f_tiles), 256, 0, stream>>>(vals, meta, No, C, (uint8_t *)packed, k_tiles);
     ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+// ---- streaming calibration: state = sumsq | lo | hi | norm (f64[C] each) | counts u32[C][bins] | chunk partials [64][C]
+CalibState carve_calib_state(void *state, int C, int bins) {
+    CalibState c{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { void *p = state ? (char *)state + off : nullptr; off += align_up(bytes, 256); return p; };
+    c.sumsq = (double *)take(sizeof(double) * C);
+    c.lo = (double *)take(sizeof(double) * C);
+    c.hi = (double *)take(sizeof(double) * C);
+    c.norm = (double *)take(sizeof(double) * C);
+    c.counts = (unsigned int *)take(sizeof(unsigned int) * (size_t)C * bins);
+    c.part_sumsq = (double *)take(sizeof(double) * 64 * (size_t)C);
+    c.part_min = (float *)take(sizeof(float) * 64 * (size_t)C);
+    c.part_max = (float *)take(sizeof(float) * 64 * (size_t)C);
+    c.total_bytes = off;
+    return c;
+}
+
+esp_status_t launch_calib_reset(const CalibState &c, int C, int bins, cudaStream_t stream) {
+    const long n = (long)C * bins;
+    calib_reset_kernel<<<ceil_div(n, 256), 256, 0, stream>>>(C, bins, c.sumsq, c.lo, c.hi, c.counts);
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+esp_status_t launch_calib_range(const CalibState &c, const __half *X, int T, int C, long ldx, cudaStream_t stream) {
+    int splits = ceil_div(T, 256);
+    if (splits > 64) splits = 64;
+    colstats_kernel<<<dim3(ceil_div(C, 256), splits), 256, 0, stream>>>(X, T, C, ldx, ceil_div(T, splits), c.part_sumsq, c.part_min,
+                                                                       c.part_max);
+    calib_merge_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, splits, c.part_sumsq, c.part_min, c.part_max, c.sumsq, c.lo, c.hi);
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+esp_status_t launch_calib_histogram(const CalibState &c, const __half *X, int T, int C, long ldx, int bins, cudaStream_t stream) {
+    DeviceInfo di;
+    esp_status_t st = device_info(&di);
+    if (st != ESP_OK) return st;
+    const int hsplits = pick_splits(T, ceil_div(C, 64), di.sm_count);
+    const size_t hsmem = sizeof(unsigned int) * 64 * (size_t)bins;
+    ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem));
+    histogram_kernel<<<dim3(ceil_div(C, 64), hsplits), 256, hsmem, stream>>>(X, T, C, ldx, ceil_div(T, hsplits), bins, c.lo, c.hi,
+                                                                             c.counts);
+    ESP_CUDA_OK(cudaGetLastError());
+    return ESP_OK;
+}
+
+esp_status_t launch_calib_finish(const CalibState &c, int C, int bins, long long T_total, const esp_prune_opts &o, double *chan_norm,
+                                 double *chan_entropy, double *chan_score, cudaStream_t stream) {
+    calib_norm_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, c.sumsq, c.norm);
+    // entropy needs a scratch output even when the caller does not want it: the chunk partials are free by now
+    double *entropy = chan_entropy ? chan_entropy : c.part_sumsq;
+    entropy_score_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, (int)T_total, bins, c.counts, c.norm, o.alpha, o.use_entropy,
+                                                               o.use_norm, nullptr, entropy, chan_score);
+    ESP_CUDA_OK(cudaGetLastError());
+    if (chan_norm) ESP_CUDA_OK(cudaMemcpyAsync(chan_norm, c.norm, sizeof(double) * C, cudaMemcpyDeviceToDevice, stream));
     return ESP_OK;
 }
 

@@ -35,6 +35,7 @@ struct GemmParams {
     int out_f32;
     int k_tiles;             // ceil(K / 128)
     int k_tiles_per_split;
+    const uint8_t *ximg;     // tiled pair kernel: permuted X as shared-memory images (written by xtile_kernel)
 };
 
 // ---------------------------------------------------------------------------------------------- PTX helpers
@@ -1170,9 +1171,30 @@ esp_status_t launch_wait_timeout_selftest(cudaStream_t stream) {
 
 static long transposed_ld(int M) { return (long)((M + 15) / 16 * 16); }
 
-size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
+// Workspace = [transposed copy of token-major X] [X images of the tiled pair kernel].  The first part is required for
+// every kernel but the gather kernel when X is token-major; the second lets large M use the tiled pair kernel.
+static size_t transpose_bytes(int M, int K, const esp_gemm_opts &o) {
     if (o.x_layout == ESP_X_CHANNEL_MAJOR || o.force_kernel == ESP_KERNEL_GATHER) return 0;
     return align_up((size_t)K * (size_t)transposed_ld(M) * 2, 256);
+}
+static size_t ximg_bytes(int M, int K, int tn) {
+    switch (tn) {
+        case 128: return xtile_bytes<128>(M, K);
+        case 192: return xtile_bytes<192>(M, K);
+        case 224: return xtile_bytes<224>(M, K);
+        default: return xtile_bytes<240>(M, K);
+    }
+}
+size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o) { return transpose_bytes(M, K, o); }
+size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
+    size_t n = transpose_bytes(M, K, o);
+    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 256 && o.split_k <= 1);
+    if (pair_possible) {
+        size_t img = 0;
+        for (int tn : {128, 192, 224, 240}) img = std::max(img, ximg_bytes(M, K, tn));
+        n += img;
+    }
+    return n;
 }
 
 // Resident capacity (in CTAs) of the streaming kernel for one configuration, cached per process.
@@ -1198,7 +1220,8 @@ static int stream_capacity_ctas(int bn, int split, int stages) {
     return clusters * split;
 }
 
-esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_workspace, GemmPlan *plan) {
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan) {
+    const bool have_workspace = workspace_bytes >= transpose_bytes(M, K, o) && (workspace_bytes > 0 || o.x_layout == ESP_X_CHANNEL_MAJOR);
     DeviceInfo di;
     esp_status_t st = device_info(&di);
     if (st != ESP_OK) return st;
@@ -1211,10 +1234,11 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
     if (o.force_kernel != ESP_KERNEL_GATHER && channel_major_available) {
         if (o.force_kernel == ESP_KERNEL_TMA) g.kernel = ESP_KERNEL_TMA;
         else if (o.force_kernel == ESP_KERNEL_PAIR) g.kernel = ESP_KERNEL_PAIR;
+        else if (o.force_kernel == ESP_KERNEL_PAIR_TILED) g.kernel = ESP_KERNEL_PAIR_TILED;
         else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
         else g.kernel = (M > 256 && o.split_k <= 1) ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;   // the pair kernel has no K-slices
     }
-    if (g.kernel == ESP_KERNEL_PAIR) {
+    if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED) {
         if (bn == 0) {
             // widest token tile unless a narrower one saves a whole wave of clusters: cost ~ waves x tile width
             const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
@@ -1226,6 +1250,10 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, bool have_wo
             }
         }
         if (bn != 128 && bn != 192 && bn != 224 && bn != 240 && bn != 256) return ESP_ERR_INVALID_ARG;
+        // the tiled form needs room for the X images behind the transposed copy; without it the gather form runs
+        const bool room = bn != 256 && workspace_bytes >= transpose_bytes(M, K, o) + ximg_bytes(M, K, bn);
+        if (g.kernel == ESP_KERNEL_PAIR_TILED && !room) return ESP_ERR_WORKSPACE;
+        if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room) g.kernel = ESP_KERNEL_PAIR_TILED;
         g.token_tile = bn;
         g.split_k = 1;
         g.stages = 0;
@@ -1308,6 +1336,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.out_f32 = (o.out_dtype == ESP_OUT_F32) ? 1 : 0;
     p.k_tiles = ceil_div(K, kTileK);
     p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
+    p.ximg = nullptr;
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
     if (plan.kernel != ESP_KERNEL_GATHER) {
         if (!p.x_channel_major) {
@@ -1322,6 +1351,20 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.x_channel_major = 1;
         }
         const bool dependent = o.static_weights != 0;
+        if (plan.kernel == ESP_KERNEL_PAIR_TILED) {
+            const size_t off = transpose_bytes(M, K, o);
+            if (!workspace || workspace_bytes < off + ximg_bytes(M, K, plan.token_tile)) return ESP_ERR_WORKSPACE;
+            uint8_t *img = reinterpret_cast<uint8_t *>(workspace) + off;
+            p.ximg = img;
+            esp_status_t st;
+            switch (plan.token_tile) {
+                case 128: st = launch_xtile<128>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
+                case 192: st = launch_xtile<192>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
+                case 224: st = launch_xtile<224>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
+                case 240: st = launch_xtile<240>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
+                default: return ESP_ERR_INVALID_ARG;
+            }
+        }
         if (plan.kernel == ESP_KERNEL_PAIR) {
             switch (plan.token_tile) {
                 case 128: return launch_pair<2, 128>(p, dependent, stream);

@@ -29,6 +29,12 @@
 //                      (four warps per quarter of the accumulator lanes)
 // A stage's `empty` barrier and the final `accum` barrier are signalled in both CTAs at once by
 // tcgen05.commit with a CTA mask.  No load uses cluster multicast.
+//
+// TILED = true is the same kernel fed differently: a pass over X (xtile_kernel) has already applied the permutation
+// and written, for every (token tile, CTA rank, 128-channel step), the exact shared-memory image of the X operand
+// (kXStage bytes, swizzled) into the caller's workspace.  A stage is then three bulk copies (two weight tiles, one X
+// image), each from lane 0 of a warp of its own; the sixteen warps no longer gather, they only run the epilogue.
+// The 16-byte gather path delivers 32 B/clk per SM, bulk copies about 70: the price is one more pass over X.
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -98,7 +104,42 @@ struct PairCfg {
     __host__ __device__ static constexpr uint32_t meta_col(int a, int buf) { return (uint32_t)a * 256u + TN + 4u * buf; }
 };
 
-template <int NA, int TN>
+// X [K, ldx] channel-major -> images of the pair kernel's X stages: image (h, kt) with h = 2 * token tile + CTA rank holds
+// channels perm[kt*128 .. +127] of tokens h's half tile, as [64-token block][128 rows][128 bytes] with the 16-byte chunk c
+// of row r stored at chunk c ^ (r & 7).  Rows beyond K and tokens beyond M are zero.  grid (k_tiles, 2 * token tiles).
+template <int TN>
+__global__ void __launch_bounds__(256) xtile_kernel(const uint16_t *__restrict__ X, long ldx, int M, int K,
+                                                    const int32_t *__restrict__ perm, uint8_t *__restrict__ img, int k_tiles) {
+    using L = PairCfg<2, TN>;
+    const int kt = blockIdx.x, h = blockIdx.y;
+    const int tok_cta = (h >> 1) * TN + (h & 1) * L::kHalf;
+    uint8_t *dst = img + ((size_t)h * k_tiles + kt) * L::kXStage;
+    grid_launch_dependents();
+    grid_dependency_wait();                  // X may be the preceding kernel's output; the images may still be read by it
+#pragma unroll 4
+    for (int idx = threadIdx.x; idx < L::kTokBlocks * 1024; idx += 256) {
+        const int cc = idx & 7, r = (idx >> 3) & 127, tb = idx >> 10;
+        const int local = tb * 64 + cc * 8, t = tok_cta + local;
+        const int kpos = kt * kTileK + r;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (kpos < K && local < L::kHalf && t < M) {
+            const int ch = perm ? __ldg(perm + kpos) : kpos;
+            const uint16_t *src = X + (long)ch * ldx + t;
+            if (t + 8 <= M) {
+                v = __ldg(reinterpret_cast<const uint4 *>(src));
+            } else {
+                uint16_t e[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) e[i] = (t + i < M) ? __ldg(src + i) : (uint16_t)0;
+                v = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16), e[4] | ((uint32_t)e[5] << 16),
+                               e[6] | ((uint32_t)e[7] << 16));
+            }
+        }
+        *reinterpret_cast<uint4 *>(dst + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+    }
+}
+
+template <int NA, int TN, bool TILED>
 __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p) {
     using L = PairCfg<NA, TN>;
     constexpr int STAGES = L::kStages;
@@ -132,7 +173,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full(s), kPairProducers + (uint32_t)n_present);    // X threads + one arrival per weight-tile copy
+            // one arrival per weight-tile copy + the X threads (gather) or the X image copy (tiled)
+            mbar_init(full(s), (TILED ? 1u : (uint32_t)kPairProducers) + (uint32_t)n_present);
             mbar_init(empty(s), 1);
             mbar_init(peer_full(s), 1);
         }
@@ -216,13 +258,41 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             tc_commit_pair(accum_bar, (uint16_t)3);
         }
     } else {
+        const int g = threadIdx.x - 64;
+        bool alive = true;
+        if constexpr (TILED) {
+            // ---- copy issuers: lane 0 of warp 2 + s * (NA + 1) + kind feeds ring slot s with weight tile `kind` (< NA) or
+            // with the X image (kind == NA); it meets every phase of its slot's `empty` barrier.  The other lanes wait at
+            // the vote below without polling.
+            constexpr int kCopies = NA + 1;
+            static_assert(kCopies * STAGES <= 16, "one issuing warp per copy of the ring");
+            const int iw = warp - 2;
+            if (lane == 0 && iw < kCopies * STAGES) {
+                const int s = iw / kCopies, kind = iw % kCopies;
+                const bool is_x = kind == NA;
+                if (is_x) {
+                    grid_dependency_wait();                               // the images are written by the preceding kernel
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
+                if (is_x || present[kind]) {
+                    const uint32_t bytes = is_x ? (uint32_t)L::kXStage : (uint32_t)kTileBytes;
+                    const uint8_t *src = is_x ? p.ximg + ((size_t)(blockIdx.y * 2 + rank) * nk) * L::kXStage
+                                              : p.packed + (long)ftile[kind] * nk * kTileBytes;
+                    const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                        mbar_arrive_expect_tx(full(s), bytes);
+                        bulk_load(dst, src + (size_t)it * bytes, bytes, full(s));
+                    }
+                }
+            }
+        } else {
         // ---- X producers: thread g copies 16-byte chunk (g & 7) of rows (g >> 3) and (g >> 3) + 64 of every 64-token
         // block.  Its two permutation entries are loaded kAhead steps early into registers (the loop is unrolled by
         // kAhead so the register ring has constant indices): the load's latency never sits between two steps.
-        const int g = threadIdx.x - 64;
         const int cc = g & 7, rg = g >> 3;
         const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
-        bool alive = true;
         constexpr int kAhead = 4;
         auto channel_of = [&](int it, int row) -> int {
             const int kpos = it * kTileK + row;
@@ -273,6 +343,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                     }
                 }
             }
+        }
         }
         // ---- epilogue: this CTA's 128 feature rows of every accumulator, all TN token columns; warp w reads lane
         // quarter w % 4 and the 16-column pieces (w - 2) / 4, + 4, + 8, ...
@@ -352,10 +423,31 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     }
 }
 
-template <int NA, int TN>
+template <int TN>
+size_t xtile_bytes(int M, int K) {
+    return (size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * PairCfg<2, TN>::kXStage;
+}
+
+template <int TN>
+esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, bool dependent, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.k_tiles, 2 * ((p.M + TN - 1) / TN), 1);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile_kernel<TN>, reinterpret_cast<const uint16_t *>(p.X), p.ldx, p.M, p.K, p.perm, img,
+                                   p.k_tiles));
+    return ESP_OK;
+}
+
+template <int NA, int TN, bool TILED = false>
 esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream) {
     using L = PairCfg<NA, TN>;
-    auto kern = spgemm_pair_kernel<NA, TN>;
+    auto kern = spgemm_pair_kernel<NA, TN, TILED>;
     ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
     const int f_tiles = (p.N + 127) / 128;
     cudaLaunchConfig_t cfg = {};

@@ -52,7 +52,7 @@ extern "C" esp_status_t esp_spgemm_static(const void *X, int M, int K, long ldx,
     esp_gemm_opts_default(&o);
     o.x_layout = ESP_X_TOKEN_MAJOR;
     o.out_dtype = out_dtype;
-    const size_t need = gemm_workspace_bytes(M, K, o);
+    const size_t need = gemm_workspace_min_bytes(M, K, o);   // the transposed copy; X images only if they fit too
     if (need > (size_t)ESP_STATIC_SCRATCH_BYTES) return ESP_ERR_STATIC_LIMIT;
     DeviceInfo di;
     esp_status_t st = device_info(&di);
@@ -62,10 +62,11 @@ extern "C" esp_status_t esp_spgemm_static(const void *X, int M, int K, long ldx,
     st = static_scratch_address(&scratch);
     if (st != ESP_OK) return st;
     GemmPlan plan;
-    st = plan_gemm(M, N, K, o, /*have_workspace=*/true, &plan);
+    st = plan_gemm(M, N, K, o, (size_t)ESP_STATIC_SCRATCH_BYTES, &plan);
     if (st != ESP_OK) return st;
     // The transposing pre-pass writes every element of the K x ceil16(M) region the GEMM reads (zeros in the
-    // padding columns), so nothing has to be cleared although the array keeps the previous call's contents.
+    // padding columns), and the tiling pass every byte of the images, so nothing has to be cleared although the
+    // array keeps the previous call's contents.
     return launch_spgemm((const __half *)X, M, K, ldx, packed, perm, N, Y, ldy, o, plan, scratch,
                          (size_t)ESP_STATIC_SCRATCH_BYTES, (cudaStream_t)cuda_stream);
 }

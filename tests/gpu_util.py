@@ -87,3 +87,32 @@ def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0
     torch.cuda.synchronize()
     assert b.esp_last_device_status() == b.ESP_OK
     return Y.cpu().numpy()
+
+
+def calibrate_in_chunks(chunks, alpha, bins=100, **opts):
+    """Streaming calibration over a list of [T_i, C] fp16 arrays; returns (norm, entropy, score, counts) on the host."""
+    dev = torch.device(DEV)
+    C = chunks[0].shape[1]
+    o = b.esp_prune_opts_default()
+    o.alpha, o.bins = alpha, bins
+    for k, v in opts.items():
+        setattr(o, k, v)
+    nbytes = b.esp_calib_state_bytes(C, bins)
+    state = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    state.fill_(0xA5)                                # reset must not depend on what the buffer held
+    dchunks = [torch.from_numpy(np.ascontiguousarray(c)).to(dev) for c in chunks]
+    b.esp_calib_reset(state, C, bins)
+    for d in dchunks:
+        b.esp_calib_range(state, d, bins)
+    for d in dchunks:
+        b.esp_calib_histogram(state, d, bins)
+    norm = torch.empty(C, dtype=torch.float64, device=dev)
+    entropy = torch.empty(C, dtype=torch.float64, device=dev)
+    score = torch.empty(C, dtype=torch.float64, device=dev)
+    T_total = sum(c.shape[0] for c in chunks)
+    b.esp_calib_finish(state, C, T_total, o, norm, entropy, score)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    off = 4 * ((8 * C + 255) // 256 * 256)
+    counts = state[off: off + 4 * C * bins].view(torch.int32).reshape(C, bins).cpu().numpy()
+    return norm.cpu().numpy(), entropy.cpu().numpy(), score.cpu().numpy(), counts, score

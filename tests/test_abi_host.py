@@ -129,3 +129,15 @@ def test_no_gpu_means_cuda_error_not_a_fallback():
     # valid arguments, no device: the call must fail loudly, never compute on the CPU
     assert prune_call() in (b.ESP_ERR_CUDA, b.ESP_ERR_UNSUPPORTED)
     assert gemm_call() in (b.ESP_ERR_CUDA, b.ESP_ERR_UNSUPPORTED)
+
+
+def test_calibration_state_size_and_argument_checks():
+    C, bins = 512, 100
+    n = b.esp_calib_state_bytes(C, bins)
+    # four fp64 vectors, the counts, and 64 chunk partials of (fp64, f32, f32) per channel
+    assert n >= 4 * 8 * C + 4 * C * bins + 64 * C * 16
+    assert n % 256 == 0
+    assert b.esp_calib_state_bytes(C + 1, bins) == 0
+    assert b.esp_calib_state_bytes(C, 1) == 0
+    assert b._lib.esp_calib_reset(None, C, bins, None) == b.ESP_ERR_INVALID_ARG
+    assert b._lib.esp_calib_range(None, None, 4, C, C, bins, None) == b.ESP_ERR_INVALID_ARG

@@ -188,3 +188,36 @@ def test_four_of_eight_pattern(No, C, T):
     with pytest.raises(b.EsparseError) as e:
         GpuPrune(W, X, alpha, stats=False, pack=True, n_keep=4, m_group=8, use_lbs=0)
     assert e.value.status == b.ESP_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("C,splits", [(264, (100, 37, 256, 3)), (1024, (77,)), (512, (1, 1, 700, 5000))])
+def test_streaming_calibration_equals_one_shot(C, splits):
+    """Chunked statistics (two passes over the chunks) against the oracle on the concatenation: counts bit-exact,
+    norm / entropy / score to the statistics bar; then the streamed score drives the same pruning decisions."""
+    from tests.gpu_util import GpuPrune, calibrate_in_chunks
+    T = sum(splits)
+    W, X = layer(900 + C, 128, C, T)
+    X[:, 5] = 3.0
+    X[-1, 7] = 1000.0                                           # the range of channel 7 is set by the last chunk
+    alpha = 1.0 / math.sqrt(T)
+    chunks, r = [], 0
+    for n in splits:
+        chunks.append(X[r: r + n]); r += n
+    norm, ent, score, counts, score_d = calibrate_in_chunks(chunks, alpha)
+    assert np.array_equal(counts, orc.channel_histogram(X))
+    assert counts.sum(axis=1).tolist() == [T] * C
+    am, ir = orc.channel_norm(X), orc.channel_entropy(X)
+    assert np.allclose(norm, am, rtol=STAT_RTOL, atol=0)
+    assert np.allclose(ent, ir, rtol=STAT_RTOL, atol=1e-14)
+    assert np.allclose(score, orc.channel_score(ir, am, alpha), rtol=STAT_RTOL, atol=0)
+    assert ent[5] == 0.0
+    # ablation switches reach the streamed score too
+    _, _, s_norm_only, _, _ = calibrate_in_chunks(chunks, alpha, use_entropy=0)
+    assert np.allclose(s_norm_only, alpha * am, rtol=STAT_RTOL, atol=0)
+    # the streamed score feeds the pruner without the calibration matrix
+    ref = orc.metric_prune(W, X, alpha, use_lbs=False, score=score, objectives=False)
+    g = GpuPrune(W, None, alpha, score=score, use_lbs=0)
+    vals, meta, perm = g.host()
+    assert np.array_equal(perm, ref.theta) or ref.near_tie_sort > 0
+    if np.array_equal(perm, ref.theta):
+        assert_masks_match(vals, meta, ref)

@@ -94,22 +94,47 @@ def test_prefill_tiled_kernels(M, N, K, kernel):
           orc.product(X, vals, meta, None))
 
 
+@pytest.mark.parametrize("kernel", [5, 6])
 @pytest.mark.parametrize("M", [130, 300, 520, 1000])
 @pytest.mark.parametrize("N,K", [(256, 512), (200, 264), (640, 1160), (1100, 384)])
-def test_prefill_pair_kernel(M, N, K):
-    """The two-SM kernel (5): feature-pair tiles with one to four of their 128-feature tiles present, ragged
-    token / feature / channel tails, every tile width, both layouts and output types."""
+def test_prefill_pair_kernel(M, N, K, kernel):
+    """The two-SM kernel, fed by the permutation gather (5) or by bulk copies of pre-tiled X images (6): feature-pair
+    tiles with one to four of their 128-feature tiles present, ragged token / feature / channel tails, every tile
+    width, both layouts and output types."""
     from tests.gpu_util import pack_on_gpu, spgemm
     vals, meta, theta = pruned(N * 5 + K + M, N, K)
     X = np.random.default_rng(M + 2).standard_normal((M, K)).astype(np.float16)
     Yref = orc.product(X, vals, meta, theta)
     packed = pack_on_gpu(vals, meta)
-    check(spgemm(X, packed, theta, N, channel_major=True, kernel=5), Yref)
-    check(spgemm(X, packed, theta, N, channel_major=True, kernel=5, out_f32=True), Yref, True)
-    for tile in (128, 192, 224, 256):
-        check(spgemm(X, packed, theta, N, channel_major=True, kernel=5, token_tile=tile, out_f32=True), Yref, True)
-    check(spgemm(X, packed, theta, N, kernel=5), Yref)                          # token-major via the transposed copy
-    check(spgemm(X, packed, None, N, channel_major=True, kernel=5), orc.product(X, vals, meta, None))
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel), Yref)
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel, out_f32=True), Yref, True)
+    for tile in (128, 192, 224) + ((256,) if kernel == 5 else ()):
+        check(spgemm(X, packed, theta, N, channel_major=True, kernel=kernel, token_tile=tile, out_f32=True), Yref, True)
+    check(spgemm(X, packed, theta, N, kernel=kernel), Yref)                     # token-major via the transposed copy
+    check(spgemm(X, packed, None, N, channel_major=True, kernel=kernel), orc.product(X, vals, meta, None))
+
+
+def test_tiled_pair_kernel_is_the_default_with_room_and_needs_it():
+    """Large M with the full workspace plans the tiled form; without room for the images the gather form; forcing the
+    tiled form without a workspace is refused; both forms give the same bits (same MMAs in the same order)."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu, spgemm
+    M, N, K = 700, 640, 1160
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    assert b.esp_spgemm_plan(M, N, K, o, True)["kernel"] == b.ESP_KERNEL_PAIR_TILED
+    assert b.esp_spgemm_plan(M, N, K, o, False)["kernel"] == b.ESP_KERNEL_PAIR
+    assert b.esp_spgemm_workspace_bytes(M, N, K, o) >= 2 * M * K
+    vals, meta, theta = pruned(4, N, K)
+    X = np.random.default_rng(8).standard_normal((M, K)).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    a = spgemm(X, packed, theta, N, channel_major=True, kernel=6, out_f32=True)
+    assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, kernel=5, out_f32=True))
+    assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, out_f32=True))
+    check(spgemm(X, packed, theta, N, channel_major=True, workspace=False), orc.product(X, vals, meta, theta))
+    with pytest.raises(b.EsparseError):
+        spgemm(X, packed, theta, N, channel_major=True, kernel=6, workspace=False)
 
 
 def test_pair_kernel_long_k_and_determinism():
@@ -171,6 +196,42 @@ def test_chain_of_dependent_launches_with_static_weights():
     torch.cuda.synchronize()
     assert b.esp_last_device_status() == b.ESP_OK
     for i in range(6):
+        check(acts[i + 1].cpu().numpy(), orc.product(acts[i].cpu().numpy(), vals, meta, theta))
+
+
+@pytest.mark.parametrize("channel_major", [False, True])
+def test_chain_of_dependent_prefill_launches(channel_major):
+    """The same for the large-M path, whose tiling pass and GEMM share one workspace from launch to launch: four layers,
+    three rounds, every launch a programmatic dependent of the one before."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    N = K = 1024
+    M = 520
+    vals, meta, theta = pruned(78, N, K)
+    vals = (vals.astype(np.float32) * 1.7).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    dev = torch.device("cuda:0")
+    th = torch.from_numpy(theta).to(dev)
+    X0 = np.random.default_rng(4).standard_normal((M, K)).astype(np.float16)
+    acts = [torch.from_numpy(X0).to(dev)] + [torch.empty(M, N, dtype=torch.float16, device=dev) for _ in range(4)]
+    o = b.esp_gemm_opts_default()
+    o.static_weights = 1
+    if channel_major:
+        o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    assert b.esp_spgemm_plan(M, N, K, o, True)["kernel"] == b.ESP_KERNEL_PAIR_TILED
+    ws = torch.empty(b.esp_spgemm_workspace_bytes(M, N, K, o), dtype=torch.uint8, device=dev)
+    xt = torch.empty(K, M, dtype=torch.float16, device=dev)
+    for rep in range(3):
+        for i in range(4):
+            if channel_major:
+                xt.copy_(acts[i].t())                                 # the hand-over in channel-major form
+                b.esp_spgemm(xt, packed, th, acts[i + 1], o, ws)
+            else:
+                b.esp_spgemm(acts[i], packed, th, acts[i + 1], o, ws)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    for i in range(4):
         check(acts[i + 1].cpu().numpy(), orc.product(acts[i].cpu().numpy(), vals, meta, theta))
 
 
