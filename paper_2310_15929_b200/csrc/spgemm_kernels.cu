@@ -36,6 +36,7 @@ struct GemmParams {
     int k_tiles;             // ceil(K / 128)
     int k_tiles_per_split;
     const uint8_t *ximg;     // tiled pair kernel: permuted X as shared-memory images (written by xtile_kernel)
+    const uint32_t *xflags;  // one word per image: 1 once it is complete
 };
 
 // ---------------------------------------------------------------------------------------------- PTX helpers
@@ -1337,6 +1338,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.k_tiles = ceil_div(K, kTileK);
     p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
     p.ximg = nullptr;
+    p.xflags = nullptr;
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
     if (plan.kernel != ESP_KERNEL_GATHER) {
         if (!p.x_channel_major) {
@@ -1355,14 +1357,23 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             const size_t off = transpose_bytes(M, K, o);
             if (!workspace || workspace_bytes < off + ximg_bytes(M, K, plan.token_tile)) return ESP_ERR_WORKSPACE;
             uint8_t *img = reinterpret_cast<uint8_t *>(workspace) + off;
+            uint32_t *flags = nullptr;
+            switch (plan.token_tile) {
+                case 128: flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<128>(M, K)); break;
+                case 192: flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<192>(M, K)); break;
+                case 224: flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<224>(M, K)); break;
+                case 240: flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<240>(M, K)); break;
+                default: return ESP_ERR_INVALID_ARG;
+            }
             p.ximg = img;
+            p.xflags = flags;
+            // The GEMM is always the tiling pass's programmatic dependent (it waits on the flags, not on the grid).
             esp_status_t st;
             switch (plan.token_tile) {
-                case 128: st = launch_xtile<128>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
-                case 192: st = launch_xtile<192>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
-                case 224: st = launch_xtile<224>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
-                case 240: st = launch_xtile<240>(p, img, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
-                default: return ESP_ERR_INVALID_ARG;
+                case 128: st = launch_xtile<128>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
+                case 192: st = launch_xtile<192>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
+                case 224: st = launch_xtile<224>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
+                default: st = launch_xtile<240>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
             }
         }
         if (plan.kernel == ESP_KERNEL_PAIR) {

@@ -30,11 +30,12 @@
 // A stage's `empty` barrier and the final `accum` barrier are signalled in both CTAs at once by
 // tcgen05.commit with a CTA mask.  No load uses cluster multicast.
 //
-// TILED = true is the same kernel fed differently: a pass over X (xtile_kernel) has already applied the permutation
-// and written, for every (token tile, CTA rank, 128-channel step), the exact shared-memory image of the X operand
-// (kXStage bytes, swizzled) into the caller's workspace.  A stage is then three bulk copies (two weight tiles, one X
-// image), each from lane 0 of a warp of its own; the sixteen warps no longer gather, they only run the epilogue.
-// The 16-byte gather path delivers 32 B/clk per SM, bulk copies about 70: the price is one more pass over X.
+// TILED = true is the same kernel fed differently: a pass over X (xtile_kernel) applies the permutation and writes,
+// for every (token tile, CTA rank, 128-channel step), the exact shared-memory image of the X operand (kXStage bytes,
+// swizzled) into the caller's workspace.  A stage is then three bulk copies (two weight tiles, one X image), each from
+// lane 0 of a warp of its own; the sixteen warps no longer gather, they only run the epilogue.  The 16-byte gather
+// path delivers 32 B/clk per SM, bulk copies about 70: the price is one more pass over X.  That pass and the GEMM run
+// concurrently: the GEMM is launched as the pass's programmatic dependent and takes each image when its flag is up.
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -68,6 +69,19 @@ __device__ __forceinline__ bool mbar_wait_1t(uint32_t bar, uint32_t parity, vola
     for (uint32_t i = 0; i < (1u << 15); ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait(bar, parity, abort_flag);
+}
+// One non-blocking look at a barrier.  The result is a register the caller reads much later: the instruction's round
+// trip (a few hundred clocks even when the phase is complete) then overlaps whatever is issued in between.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
 }
 __device__ __forceinline__ bool mbar_wait_cluster_1t(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     for (uint32_t i = 0; i < (1u << 15); ++i) {
@@ -106,37 +120,84 @@ struct PairCfg {
 
 // X [K, ldx] channel-major -> images of the pair kernel's X stages: image (h, kt) with h = 2 * token tile + CTA rank holds
 // channels perm[kt*128 .. +127] of tokens h's half tile, as [64-token block][128 rows][128 bytes] with the 16-byte chunk c
-// of row r stored at chunk c ^ (r & 7).  Rows beyond K and tokens beyond M are zero.  grid (k_tiles, 2 * token tiles).
+// of row r stored at chunk c ^ (r & 7).  Rows beyond K and tokens beyond M are zero.  grid (2 * token tiles, k_tiles):
+// early channel steps of every token tile first, the order the GEMM consumes them in.
+//
+// flags[h * k_tiles + kt] goes 0 -> 1 when image (h, kt) is complete.  The dependent GEMM may start once every CTA
+// here has passed griddepcontrol.launch_dependents, which each CTA issues only after it has lowered its own flag (left
+// up by the previous call, or garbage in a fresh workspace): the GEMM never sees a stale 1.
 template <int TN>
 __global__ void __launch_bounds__(256) xtile_kernel(const uint16_t *__restrict__ X, long ldx, int M, int K,
-                                                    const int32_t *__restrict__ perm, uint8_t *__restrict__ img, int k_tiles) {
+                                                    const int32_t *__restrict__ perm, uint8_t *__restrict__ img,
+                                                    uint32_t *__restrict__ flags, int k_tiles) {
     using L = PairCfg<2, TN>;
-    const int kt = blockIdx.x, h = blockIdx.y;
+    const int h = blockIdx.x, kt = blockIdx.y;
     const int tok_cta = (h >> 1) * TN + (h & 1) * L::kHalf;
     uint8_t *dst = img + ((size_t)h * k_tiles + kt) * L::kXStage;
-    grid_launch_dependents();
-    grid_dependency_wait();                  // X may be the preceding kernel's output; the images may still be read by it
-#pragma unroll 4
-    for (int idx = threadIdx.x; idx < L::kTokBlocks * 1024; idx += 256) {
-        const int cc = idx & 7, r = (idx >> 3) & 127, tb = idx >> 10;
-        const int local = tb * 64 + cc * 8, t = tok_cta + local;
-        const int kpos = kt * kTileK + r;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (kpos < K && local < L::kHalf && t < M) {
-            const int ch = perm ? __ldg(perm + kpos) : kpos;
-            const uint16_t *src = X + (long)ch * ldx + t;
-            if (t + 8 <= M) {
-                v = __ldg(reinterpret_cast<const uint4 *>(src));
-            } else {
-                uint16_t e[8];
+    uint32_t *flag = flags + (size_t)h * k_tiles + kt;
+    // thread -> chunk cc = tid & 7 of rows (tid >> 3) + 32 * i; its permutation entries do not depend on the preceding
+    // kernel, and all of its row loads are in flight together
+    const int cc = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+    int ch[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) e[i] = (t + i < M) ? __ldg(src + i) : (uint16_t)0;
-                v = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16), e[4] | ((uint32_t)e[5] << 16),
-                               e[6] | ((uint32_t)e[7] << 16));
+    for (int i = 0; i < 4; ++i) {
+        const int kpos = kt * kTileK + r0 + 32 * i;
+        ch[i] = kpos < K ? (perm ? __ldg(perm + kpos) : kpos) : -1;
+    }
+    grid_dependency_wait();                  // X may be the preceding kernel's output; the images may still be read by it
+    if (threadIdx.x == 0) {
+        asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(0u) : "memory");
+        __threadfence();
+    }
+    __syncthreads();
+    grid_launch_dependents();
+    uint4 v[4][L::kTokBlocks];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int tb = 0; tb < L::kTokBlocks; ++tb) {
+            const int local = tb * 64 + cc * 8, t = tok_cta + local;
+            v[i][tb] = make_uint4(0u, 0u, 0u, 0u);
+            if (ch[i] >= 0 && local < L::kHalf && t < M) {
+                const uint16_t *src = X + (long)ch[i] * ldx + t;
+                if (t + 8 <= M) {
+                    v[i][tb] = __ldg(reinterpret_cast<const uint4 *>(src));
+                } else {
+                    uint16_t e[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) e[j] = (t + j < M) ? __ldg(src + j) : (uint16_t)0;
+                    v[i][tb] = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
+                                          e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
+                }
             }
         }
-        *reinterpret_cast<uint4 *>(dst + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = r0 + 32 * i;
+#pragma unroll
+        for (int tb = 0; tb < L::kTokBlocks; ++tb)
+            *reinterpret_cast<uint4 *>(dst + tb * 16384 + r * 128 + ((cc ^ (r & 7)) << 4)) = v[i][tb];
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
+}
+
+// Bounded wait for an image flag (set by a CTA of the tiling pass that is resident before this kernel can start).
+__device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v == 1u) return true;
+        if (i > 8) {
+            if (*abort_flag) return false;
+            __nanosleep(128);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
+    return false;
 }
 
 template <int NA, int TN, bool TILED>
@@ -149,7 +210,6 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const uint32_t bar_base = sbase + L::kBarOff;
     auto full = [&](int s) { return bar_base + 8u * s; };
     auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
-    auto peer_full = [&](int s) { return bar_base + 8u * (16 + s); };    // used in the leader only
     const uint32_t accum_bar = bar_base + 8u * 24;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
@@ -173,10 +233,10 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            // one arrival per weight-tile copy + the X threads (gather) or the X image copy (tiled)
-            mbar_init(full(s), (TILED ? 1u : (uint32_t)kPairProducers) + (uint32_t)n_present);
+            // one arrival per weight-tile copy + the X threads (gather) or the X image copy (tiled); the leader's barrier
+            // also takes rank 1's "my stage has landed", so the MMA thread waits on one barrier per step
+            mbar_init(full(s), (TILED ? 1u : (uint32_t)kPairProducers) + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
             mbar_init(empty(s), 1);
-            mbar_init(peer_full(s), 1);
         }
         mbar_init(accum_bar, 1);
         *abort_flag = 0;
@@ -209,8 +269,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                 if (!mbar_wait_1t(full(s), ph, abort_flag)) break;
-                fence_async_smem();          // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
-                mbar_arrive_remote(map_to_rank(peer_full(s), 0));
+                if (!TILED) fence_async_smem();   // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
+                mbar_arrive_remote(map_to_rank(full(s), 0));
             }
         } else if (lane == 0) {
             // One thread issues every MMA of the pair, so its own instruction stream must stay far shorter than the
@@ -229,6 +289,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             for (int j = 0; j < 4; ++j) bd0[j] = smem_desc(sbase + L::kWStage + j * 4096, 16384, 1024, kLayoutSw128);
             constexpr int kUnroll = STAGES * 2;                           // ring slot and metadata buffer both periodic
             bool alive = true;
+            uint32_t seen = 0;                                            // the next step's barrier was seen complete
             for (int it0 = 0; it0 < nk && alive; it0 += kUnroll) {
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
@@ -236,9 +297,16 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                     if (it >= nk) break;
                     const int s = u % STAGES;                             // == it % STAGES (it0 is a multiple of STAGES)
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                    if (!mbar_wait_1t(full(s), ph, abort_flag)) { alive = false; break; }
-                    if (!mbar_wait_cluster_1t(peer_full(s), ph, abort_flag)) { alive = false; break; }
-                    fence_async_smem();
+                    uint32_t seen_a = 0, seen_b = 0;
+                    const uint32_t nbar = full((u + 1) % STAGES), nph = (uint32_t)((it + 1) / STAGES) & 1u;
+                    // Rank 1's arrival only relays that its stage is complete: one barrier for both CTAs, no cluster-scope
+                    // acquire; a proxy fence only where the rows were written by cp.async.  A wait costs this thread ~300 clocks even
+                    // when the phase is complete -- with the ~700 it needs to issue a step's MMAs that is more than the 960
+                    // they run -- so the next step's barrier is looked at without blocking while this step is being issued,
+                    // and waited on only if not seen yet.
+                    if (!seen && !mbar_wait_1t(full(s), ph, abort_flag)) { alive = false; break; }
+                    if (!TILED) fence_async_smem();
+                    if (it + 1 < nk) seen_a = mbar_test(nbar, nph);
                     tc_fence_after();
                     const uint64_t soff = (uint64_t)((uint32_t)(s * L::kStage) >> 4);   // added to the address field
 #pragma unroll
@@ -251,8 +319,10 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                             tc_mma_sparse_f16_pair(tmem + L::acc_col(a), ad0[a][j] + soff, bd0[j] + soff, tmem + (col & ~1u),
                                                    idesc | (col & 1u), (it > 0 || j > 0) ? 1u : 0u);
                         }
+                        if (it + 1 < nk) seen_b |= mbar_test(nbar, nph);
                     }
                     tc_commit_pair(empty(s), (uint16_t)3);
+                    seen = seen_a | seen_b;
                 }
             }
             tc_commit_pair(accum_bar, (uint16_t)3);
@@ -265,15 +335,12 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // with the X image (kind == NA); it meets every phase of its slot's `empty` barrier.  The other lanes wait at
             // the vote below without polling.
             constexpr int kCopies = NA + 1;
-            static_assert(kCopies * STAGES <= 16, "one issuing warp per copy of the ring");
+            static_assert(kCopies * STAGES <= 15, "one issuing warp per copy of the ring; warp 17 polls the accumulator barrier");
             const int iw = warp - 2;
             if (lane == 0 && iw < kCopies * STAGES) {
                 const int s = iw / kCopies, kind = iw % kCopies;
                 const bool is_x = kind == NA;
-                if (is_x) {
-                    grid_dependency_wait();                               // the images are written by the preceding kernel
-                    asm volatile("fence.proxy.async;" ::: "memory");
-                }
+                const uint32_t *xflag = p.xflags + (size_t)(blockIdx.y * 2 + rank) * nk;
                 if (is_x || present[kind]) {
                     const uint32_t bytes = is_x ? (uint32_t)L::kXStage : (uint32_t)kTileBytes;
                     const uint8_t *src = is_x ? p.ximg + ((size_t)(blockIdx.y * 2 + rank) * nk) * L::kXStage
@@ -281,6 +348,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                     const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
                     for (int it = s; it < nk; it += STAGES) {
                         const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (is_x) {
+                            // the image is written by the tiling pass while this kernel runs: wait for its flag (long up,
+                            // except in the first steps) before the slot's own wait, then order the generic-proxy writes
+                            // just acquired before this thread's asynchronous-proxy read
+                            if (!xflag_wait(xflag + it, abort_flag)) { alive = false; break; }
+                            asm volatile("fence.proxy.async;" ::: "memory");
+                        }
                         if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
                         mbar_arrive_expect_tx(full(s), bytes);
                         bulk_load(dst, src + (size_t)it * bytes, bytes, full(s));
@@ -350,7 +424,14 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         const int quarter = warp & 3;
         const int cgrp = (warp - 2) >> 2;
         const int f_local = quarter * 32 + lane;
-        const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait_cluster(accum_bar, 0, abort_flag)));
+        // One thread polls the accumulator barrier; the other 511 sleep on a named barrier meanwhile (in the tiled form
+        // most of them are idle for the whole main loop, and hundreds of polling lanes slow every other barrier down).
+        if (!alive) *abort_flag = 1;
+        __syncwarp();
+        if (warp == 17 && lane == 0 && nk > 0) (void)mbar_wait_cluster(accum_bar, 0, abort_flag);
+        __syncwarp();
+        asm volatile("bar.sync 1, %0;" ::"n"(kPairProducers) : "memory");
+        const bool ok = *abort_flag == 0;
         tc_fence_after();
         const bool y_vec = (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
         // accumulator a -> shared memory [token][128 features] in the output type -> 16-byte stores along the features.
@@ -424,14 +505,18 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 }
 
 template <int TN>
-size_t xtile_bytes(int M, int K) {
+size_t xtile_image_bytes(int M, int K) {
     return (size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * PairCfg<2, TN>::kXStage;
+}
+template <int TN>
+size_t xtile_bytes(int M, int K) {           // images + one flag word per image
+    return xtile_image_bytes<TN>(M, K) + align_up((size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * 4, 256);
 }
 
 template <int TN>
-esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, bool dependent, cudaStream_t stream) {
+esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, uint32_t *flags, bool dependent, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.k_tiles, 2 * ((p.M + TN - 1) / TN), 1);
+    cfg.gridDim = dim3(2 * ((p.M + TN - 1) / TN), p.k_tiles, 1);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -440,7 +525,7 @@ esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, bool dependent, cud
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
     ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile_kernel<TN>, reinterpret_cast<const uint16_t *>(p.X), p.ldx, p.M, p.K, p.perm, img,
-                                   p.k_tiles));
+                                   flags, p.k_tiles));
     return ESP_OK;
 }
 
