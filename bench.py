@@ -32,9 +32,9 @@ import numpy as np
 
 PREFILL_M = 2048
 DECODE_M = 16
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the 4096 x 4096 linear, from the ncu captures summarised
+# dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch on the 4096 x 4096 linear, from the ncu captures summarised
 # under profiles/ (None = the kernel changed since the counters were taken)
-PREFILL_TRAFFIC_BYTES = 36.2e6
+PREFILL_TRAFFIC_BYTES = 38.6e6
 DECODE_TRAFFIC_BYTES = 19.07e6
 WORKLOAD = 1          # llama-7b-layer
 
@@ -264,7 +264,25 @@ def run_ours(args):
     sampler = ClockSampler(local)
     sampler.start()                           # nvidia-smi needs a moment before its first sample
     pws = make_ws(PREFILL_M, po)
-    step = lambda: gemm_step(xs, ys, po, pws)
+    eager_step = lambda: gemm_step(xs, ys, po, pws)
+    # One step = the layer's seven esp_spgemm calls (each a tiling pass over X + the GEMM), recorded once into a CUDA graph
+    # and replayed: the launches then follow each other without host gaps.  --eager times the plain calls instead.
+    launches_per_step = sum(2 if b.esp_spgemm_plan(PREFILL_M, lin["N"], lin["K"], po, pws is not None)["kernel"]
+                            == b.ESP_KERNEL_PAIR_TILED else 1 for lin in layer)
+    if args.eager:
+        step = eager_step
+    else:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for _ in range(2):
+                eager_step()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                eager_step()
+        torch.cuda.synchronize()
+        step = graph.replay
     for _ in range(args.warmup):
         step()
     if dist:
@@ -438,11 +456,12 @@ def run_ours(args):
                        "M": PREFILL_M, "x_layout": args.x_layout, "accumulate": "f32", "out": "f16", "static_weights": 1,
                        "l2": "inputs larger than L2: 228 MB of distinct compressed weights + 117 MB of X + 145 MB of Y per step",
                        "replicas": "one independent layer per GPU, no collective"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 7 * args.steps,
-            "kernel": "spgemm_pair_kernel<2,240>: 7 launches per step, one per linear",
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "kernel": f"xtile_kernel + spgemm_pair_kernel<2,TN,tiled> per linear: {launches_per_step} launches per step, "
+                      + ("plain calls" if args.eager else "replayed from one CUDA graph per step"),
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": sparse_peak, "unit": "TFLOP/s",
                          "frac": achieved / sparse_peak, "traffic": PREFILL_TRAFFIC_BYTES,
-                         "note": f"dense-equivalent flops of the 7 launches of a step / their CUDA-event time; peak = 2 x "
+                         "note": f"dense-equivalent flops of a step (seven linears) / its CUDA-event time; peak = 2 x "
                                  f"{peaks['source']} burst dense bf16 ({peaks['bf16_burst']}); frac of nominal 4500 = "
                                  f"{achieved / 4500.0:.3f}; traffic = DRAM bytes of one 4096x4096 launch from the ncu "
                                  f"capture in profiles/"},
@@ -489,8 +508,11 @@ def run_profile_case(args):
     X = torch.randn(K, M, device=dev).half()
     Y = torch.empty(M, N, dtype=torch.float16, device=dev)
     o = b.esp_gemm_opts_default(); o.x_layout = b.ESP_X_CHANNEL_MAJOR
-    ms = time_steps(lambda: b.esp_spgemm(X, packed, perm, Y, o), 3, 3)
-    print(json.dumps({"case": case, "M": M, "N": N, "K": K, "ms_per_launch": ms,
+    nws = b.esp_spgemm_workspace_bytes(M, N, K, o)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws else None
+    ms = time_steps(lambda: b.esp_spgemm(X, packed, perm, Y, o, ws), 3, 3)
+    print(json.dumps({"case": case, "M": M, "N": N, "K": K, "plan": b.esp_spgemm_plan(M, N, K, o, ws is not None),
+                      "ms_per_call": ms,
                       "tflops": 2.0 * M * N * K / ms / 1e9, "gbs": gemm_bytes(M, N, K) / ms / 1e6}))
 
 
@@ -525,6 +547,8 @@ def run_table5(args):
         o = b.esp_gemm_opts_default()
         o.x_layout = b.ESP_X_CHANNEL_MAJOR
         o.static_weights = 1
+        nws = b.esp_spgemm_workspace_bytes(M, N, K, o)
+        ws = torch.empty(nws, dtype=torch.uint8, device=dev) if nws else None
         Wd = [torch.randn(N, K, device=dev).half() for _ in range(ncopies)]
         Xt = X.t().contiguous()
         reps = 4 if M > 256 else 2 * ncopies
@@ -549,15 +573,15 @@ def run_table5(args):
                 e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
                 best = min(best, e0.elapsed_time(e1) / reps)
             return best
-        ms = timed(lambda i: b.esp_spgemm(X, packs[i % ncopies], perm, Y, o))
+        ms = timed(lambda i: b.esp_spgemm(X, packs[i % ncopies], perm, Y, o, ws))
         dms = timed(lambda i: torch.matmul(Xt, Wd[i % ncopies].t()))
         assert b.esp_last_device_status() == b.ESP_OK
         print(json.dumps({"table5": name, "M": M, "N": N, "K": K, "sparse_ms": ms, "dense_cublas_ms": dms,
                           "speedup_vs_dense": dms / ms, "tflops_dense_equivalent": 2.0 * M * N * K / ms / 1e9,
-                          "gbs": gemm_bytes(M, N, K) / ms / 1e6, "plan": b.esp_spgemm_plan(M, N, K, o),
+                          "gbs": gemm_bytes(M, N, K) / ms / 1e6, "plan": b.esp_spgemm_plan(M, N, K, o, ws is not None),
                           "paper_a100_dense_ms": paper_dense_ms, "paper_a100_sparse_ms": paper_sparse_ms,
                           "paper_speedup": paper_dense_ms / paper_sparse_ms}), flush=True)
-        del packs, Wd, X, Y, Xt
+        del packs, Wd, X, Y, Xt, ws
 
 
 def main():
@@ -571,6 +595,7 @@ def main():
     ap.add_argument("--lbs-max-swaps", type=int, default=0,
                     help="cap on block-shuffle swaps per block while preparing the weights (0 = run to the end)")
     ap.add_argument("--cpu-rows", type=int, default=256)
+    ap.add_argument("--eager", action="store_true", help="time plain esp_spgemm calls instead of a CUDA graph of the step")
     ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "prune"],
                     help="run a few launches of one small case (for ncu) instead of the benchmark")
     ap.add_argument("--table5", action="store_true", help="time the GEMM shapes of the paper's Table 5 instead of the benchmark")

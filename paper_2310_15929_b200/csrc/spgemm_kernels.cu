@@ -1071,15 +1071,10 @@ int stream_cluster_capacity(int split, int stages) {
     return clusters;
 }
 
-#include "spgemm_pair.cuh"
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// Tensor map over channel-major X: dim 0 = tokens (contiguous), dim 1 = channels (ldx apart); box = 64 tokens
-// x 1 row (the row-gather form loads four such rows per instruction), 128-byte swizzle, zero fill outside.
-inline esp_status_t make_x_tensor_map(const __half *X, int M, int K, long ldx, CUtensorMap *map) {
+inline esp_status_t tensor_map_encoder(EncodeTiledFn *out) {
     static EncodeTiledFn encode = nullptr;
     if (!encode) {
         void *fn = nullptr;
@@ -1088,6 +1083,18 @@ inline esp_status_t make_x_tensor_map(const __half *X, int M, int K, long ldx, C
             return ESP_ERR_CUDA;
         encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    *out = encode;
+    return ESP_OK;
+}
+
+#include "spgemm_pair.cuh"
+
+// Tensor map over channel-major X: dim 0 = tokens (contiguous), dim 1 = channels (ldx apart); box = 64 tokens
+// x 1 row (the row-gather form loads four such rows per instruction), 128-byte swizzle, zero fill outside.
+inline esp_status_t make_x_tensor_map(const __half *X, int M, int K, long ldx, CUtensorMap *map) {
+    EncodeTiledFn encode = nullptr;
+    esp_status_t est = tensor_map_encoder(&encode);
+    if (est != ESP_OK) return est;
     cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)K};
     cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
     cuuint32_t box[2] = {64, 1};

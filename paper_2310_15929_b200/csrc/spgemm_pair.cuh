@@ -70,6 +70,18 @@ __device__ __forceinline__ bool mbar_wait_1t(uint32_t bar, uint32_t parity, vola
         if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait(bar, parity, abort_flag);
 }
+// Tiled load of a [rows x 1024-byte] box of a tensor seen as rows of 256 32-bit words, for a CTA pair: the bytes land in
+// this CTA's shared memory, their count is reported to `bar`, a shared::cluster address that may lie in the peer CTA
+// (.cta_group::2).  No cluster multicast.  The first coordinate is 0: always 16-byte aligned.
+__device__ __forceinline__ void tma_rows_pair(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(0), "r"(row), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
 // One non-blocking look at a barrier.  The result is a register the caller reads much later: the instruction's round
 // trip (a few hundred clocks even when the phase is complete) then overlaps whatever is issued in between.
 __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
@@ -201,7 +213,8 @@ __device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *a
 }
 
 template <int NA, int TN, bool TILED>
-__global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p) {
+__global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap wmap,
+                                                                      const __grid_constant__ CUtensorMap xmap) {
     using L = PairCfg<NA, TN>;
     constexpr int STAGES = L::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -223,19 +236,22 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const int f_tiles = (p.N + 127) / 128;
     int ftile[NA];
     bool present[NA];
-    int n_present = 0;
+    int n_present = 0, n_present_peer = 0;
 #pragma unroll
     for (int a = 0; a < NA; ++a) {
         ftile[a] = pair_idx * (2 * NA) + 2 * a + (int)rank;               // MMA a: rows 0..127 from rank 0, 128..255 from rank 1
         present[a] = ftile[a] < f_tiles;
         n_present += present[a] ? 1 : 0;
+        n_present_peer += (pair_idx * (2 * NA) + 2 * a + 1 - (int)rank) < f_tiles ? 1 : 0;
     }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            // one arrival per weight-tile copy + the X threads (gather) or the X image copy (tiled); the leader's barrier
-            // also takes rank 1's "my stage has landed", so the MMA thread waits on one barrier per step
-            mbar_init(full(s), (TILED ? 1u : (uint32_t)kPairProducers) + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
+            // The MMA thread waits on one barrier per step, the leader's.  Gather form: one arrival per weight-tile copy +
+            // the X threads, + rank 1's relayed "my stage has landed".  Tiled form: every copy of BOTH CTAs arrives on it
+            // and reports its bytes to it directly (rank 1's own `full` barriers stay unused).
+            mbar_init(full(s), TILED ? 2u + (uint32_t)n_present + (uint32_t)n_present_peer
+                                     : (uint32_t)kPairProducers + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
             mbar_init(empty(s), 1);
         }
         mbar_init(accum_bar, 1);
@@ -264,8 +280,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         // idle: keeps the producer warps at indices 2..17 (tensor-memory lane quarter = warp index % 4)
     } else if (warp == 1) {
         if (lane == 0 && rank != 0) {
-            // forward "my operands of this stage have landed" to the leader
-            for (int it = 0; it < nk; ++it) {
+            // gather form: forward "my operands of this stage have landed" to the leader
+            for (int it = 0; it < (TILED ? 0 : nk); ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                 if (!mbar_wait_1t(full(s), ph, abort_flag)) break;
@@ -343,9 +359,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 const uint32_t *xflag = p.xflags + (size_t)(blockIdx.y * 2 + rank) * nk;
                 if (is_x || present[kind]) {
                     const uint32_t bytes = is_x ? (uint32_t)L::kXStage : (uint32_t)kTileBytes;
-                    const uint8_t *src = is_x ? p.ximg + ((size_t)(blockIdx.y * 2 + rank) * nk) * L::kXStage
-                                              : p.packed + (long)ftile[kind] * nk * kTileBytes;
+                    constexpr int kRowBytes = 1024;                       // the tensor maps see both buffers as 1024-byte rows
+                    const CUtensorMap *map = is_x ? &xmap : &wmap;
+                    const int row0 = is_x ? (int)((blockIdx.y * 2 + rank) * nk) * (L::kXStage / kRowBytes)
+                                          : ftile[kind] * nk * (kTileBytes / kRowBytes);
+                    const int row_step = (int)bytes / kRowBytes;
                     const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
+                    const uint32_t lead_full = map_to_rank(full(s), 0);
                     for (int it = s; it < nk; it += STAGES) {
                         const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                         if (is_x) {
@@ -356,8 +376,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                             asm volatile("fence.proxy.async;" ::: "memory");
                         }
                         if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
-                        mbar_arrive_expect_tx(full(s), bytes);
-                        bulk_load(dst, src + (size_t)it * bytes, bytes, full(s));
+                        mbar_arrive_expect_tx_cluster(lead_full, bytes);
+                        tma_rows_pair(dst, map, row0 + it * row_step, lead_full);
                     }
                 }
             }
@@ -529,6 +549,21 @@ esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, uint32_t *flags, bo
     return ESP_OK;
 }
 
+// Tensor map over a linear buffer seen as rows of 1024 bytes (256 32-bit words); box = box_rows whole rows, no swizzle.
+inline esp_status_t make_rows_tensor_map(const void *base, size_t bytes, int box_rows, CUtensorMap *map) {
+    EncodeTiledFn encode = nullptr;
+    esp_status_t st = tensor_map_encoder(&encode);
+    if (st != ESP_OK) return st;
+    cuuint64_t dims[2] = {256, (cuuint64_t)(bytes / 1024)};
+    cuuint64_t strides[1] = {1024};
+    cuuint32_t box[2] = {256, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? ESP_OK : ESP_ERR_CUDA;
+}
+
 template <int NA, int TN, bool TILED = false>
 esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream) {
     using L = PairCfg<NA, TN>;
@@ -549,6 +584,14 @@ esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t strea
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 2 : 1;
-    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p));
+    CUtensorMap wmap, xmap;
+    memset(&wmap, 0, sizeof(wmap));
+    memset(&xmap, 0, sizeof(xmap));
+    if constexpr (TILED) {
+        esp_status_t st = make_rows_tensor_map(p.packed, (size_t)f_tiles * p.k_tiles * kTileBytes, kTileBytes / 1024, &wmap);
+        if (st == ESP_OK) st = make_rows_tensor_map(p.ximg, xtile_image_bytes<TN>(p.M, p.K), L::kXStage / 1024, &xmap);
+        if (st != ESP_OK) return st;
+    }
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, wmap, xmap));
     return ESP_OK;
 }
