@@ -1348,7 +1348,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.xflags = nullptr;
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
     if (plan.kernel != ESP_KERNEL_GATHER) {
-        if (!p.x_channel_major) {
+        if (!p.x_channel_major && plan.kernel != ESP_KERNEL_PAIR_TILED) {
             // token-major input: transposed (not permuted) copy into the caller's workspace
             const long ldt = transposed_ld(M);
             if (!workspace || workspace_bytes < (size_t)K * ldt * 2) return ESP_ERR_WORKSPACE;
@@ -1376,6 +1376,15 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.xflags = flags;
             // The GEMM is always the tiling pass's programmatic dependent (it waits on the flags, not on the grid).
             esp_status_t st;
+            if (!p.x_channel_major) {        // token-major: one transposing tiling pass, no transposed copy
+                const uint16_t *xt = reinterpret_cast<const uint16_t *>(X);
+                switch (plan.token_tile) {
+                    case 128: st = launch_xtile_tm<128>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
+                    case 192: st = launch_xtile_tm<192>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
+                    case 224: st = launch_xtile_tm<224>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
+                    default: st = launch_xtile_tm<240>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
+                }
+            }
             switch (plan.token_tile) {
                 case 128: st = launch_xtile<128>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
                 case 192: st = launch_xtile<192>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);

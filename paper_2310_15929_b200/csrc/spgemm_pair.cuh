@@ -196,6 +196,86 @@ __global__ void __launch_bounds__(256) xtile_kernel(const uint16_t *__restrict__
     if (threadIdx.x == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
 }
 
+// ---- token-major X: the same images straight from X [M, ldx], one pass instead of a transposed copy plus the pass above.
+// A CTA reads 64 tokens x 64 consecutive channels (128 contiguous bytes per token), transposes them in shared memory and
+// writes, for each of its channels c, the 128-byte image row of position inv[c] in the permuted order (a whole swizzled
+// row: 64 tokens).  An image gets rows from every channel group, so completion is counted per half tile h: the CTA that
+// finishes h raises all of h's flags.  xtile_prep_kernel inverts the permutation and clears flags and counters first.
+__global__ void xtile_prep_kernel(const int32_t *__restrict__ perm, int K, int32_t *__restrict__ inv, uint32_t *__restrict__ flags,
+                                  int n_flags, uint32_t *__restrict__ counts, int n_counts) {
+    grid_dependency_wait();                  // a preceding GEMM on this workspace may still be reading its flags
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < K) inv[perm ? __ldg(perm + i) : i] = i;
+    if (i < n_flags) flags[i] = 0u;
+    if (i < n_counts) counts[i] = 0u;
+}
+
+template <int TN>
+__global__ void __launch_bounds__(256) xtile_tm_kernel(const uint16_t *__restrict__ X, long ldx, int M, int K,
+                                                       const int32_t *__restrict__ inv, uint8_t *__restrict__ img,
+                                                       uint32_t *__restrict__ flags, uint32_t *__restrict__ counts, int k_tiles) {
+    using L = PairCfg<2, TN>;
+    __shared__ uint32_t s[64][33];           // [channel][token pair], one word of padding per row
+    __shared__ int s_last;
+    const int h = blockIdx.x, tb = blockIdx.y, c0 = blockIdx.z * 64;
+    const int tok_cta = (h >> 1) * TN + (h & 1) * L::kHalf;
+    grid_dependency_wait();                  // inv, the cleared flags and X itself come from preceding kernels
+    grid_launch_dependents();                // the GEMM may start: every flag it can see now is 0 or freshly raised
+    uint16_t *s16 = reinterpret_cast<uint16_t *>(&s[0][0]);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int idx = threadIdx.x + 256 * j;
+        const int chunk = idx & 7, tok = idx >> 3;
+        const int local = tb * 64 + tok, t = tok_cta + local, c = c0 + chunk * 8;
+        uint16_t e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) e[i] = 0;
+        if (local < L::kHalf && t < M && c < K) {
+            const uint16_t *src = X + (long)t * ldx + c;
+            if (c + 8 <= K) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+                e[0] = (uint16_t)v.x; e[1] = (uint16_t)(v.x >> 16); e[2] = (uint16_t)v.y; e[3] = (uint16_t)(v.y >> 16);
+                e[4] = (uint16_t)v.z; e[5] = (uint16_t)(v.z >> 16); e[6] = (uint16_t)v.w; e[7] = (uint16_t)(v.w >> 16);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) if (c + i < K) e[i] = __ldg(src + i);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s16[(chunk * 8 + i) * 66 + tok] = e[i];
+    }
+    __syncthreads();
+    uint8_t *base = img + (size_t)h * k_tiles * L::kXStage + tb * 16384;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int idx = threadIdx.x + 256 * j;
+        const int cc = idx & 7, ch = idx >> 3;
+        const int c = c0 + ch;
+        if (c < K) {
+            const int q = __ldg(inv + c), kt = q >> 7, r = q & 127;
+            const uint4 v = make_uint4(s[ch][cc * 4], s[ch][cc * 4 + 1], s[ch][cc * 4 + 2], s[ch][cc * 4 + 3]);
+            *reinterpret_cast<uint4 *>(base + (size_t)kt * L::kXStage + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+        }
+    }
+    if (blockIdx.z == gridDim.z - 1) {       // rows of the last channel step beyond K
+        for (int idx = threadIdx.x; idx < (k_tiles * kTileK - K) * 8; idx += 256) {
+            const int cc = idx & 7, q = K + (idx >> 3), r = q & 127;
+            *reinterpret_cast<uint4 *>(base + (size_t)(q >> 7) * L::kXStage + r * 128 + ((cc ^ (r & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t done = atomicAdd(counts + h, 1u) + 1u;
+        s_last = done == gridDim.y * gridDim.z;
+        if (s_last) __threadfence();
+    }
+    __syncthreads();
+    if (s_last)
+        for (int kt = threadIdx.x; kt < k_tiles; kt += 256)
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flags + (size_t)h * k_tiles + kt), "r"(1u) : "memory");
+}
+
 // Bounded wait for an image flag (set by a CTA of the tiling pass that is resident before this kernel can start).
 __device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
@@ -529,8 +609,39 @@ size_t xtile_image_bytes(int M, int K) {
     return (size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * PairCfg<2, TN>::kXStage;
 }
 template <int TN>
-size_t xtile_bytes(int M, int K) {           // images + one flag word per image
-    return xtile_image_bytes<TN>(M, K) + align_up((size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * 4, 256);
+size_t xtile_flag_bytes(int M, int K) {
+    return align_up((size_t)2 * ((M + TN - 1) / TN) * ((K + kTileK - 1) / kTileK) * 4, 256);
+}
+template <int TN>
+size_t xtile_bytes(int M, int K) {           // images | one flag word per image | inverse permutation | one counter per half tile
+    return xtile_image_bytes<TN>(M, K) + xtile_flag_bytes<TN>(M, K) + align_up((size_t)K * 4, 256) +
+           align_up((size_t)2 * ((M + TN - 1) / TN) * 4, 256);
+}
+
+// Token-major X: inverse permutation and cleared flags, then the transposing tiling pass.
+template <int TN>
+esp_status_t launch_xtile_tm(const GemmParams &p, const uint16_t *X_tm, long ldx_tm, uint8_t *img, uint32_t *flags,
+                             bool dependent, cudaStream_t stream) {
+    using L = PairCfg<2, TN>;
+    const int n_h = 2 * ((p.M + TN - 1) / TN), n_flags = n_h * p.k_tiles;
+    int32_t *inv = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(flags) + xtile_flag_bytes<TN>(p.M, p.K));
+    uint32_t *counts = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(inv) + align_up((size_t)p.K * 4, 256));
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    const int n = std::max(p.K, std::max(n_flags, n_h));
+    cfg.gridDim = dim3((n + 255) / 256, 1, 1);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile_prep_kernel, p.perm, p.K, inv, flags, n_flags, counts, n_h));
+    cfg.gridDim = dim3(n_h, L::kTokBlocks, (p.K + 63) / 64);
+    cfg.numAttrs = 1;                        // always a programmatic dependent of the preparation kernel
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile_tm_kernel<TN>, X_tm, ldx_tm, p.M, p.K, (const int32_t *)inv, img, flags, counts,
+                                   p.k_tiles));
+    return ESP_OK;
 }
 
 template <int TN>
