@@ -322,11 +322,31 @@ def run_ours(args):
         hx = [h.t().contiguous().pin_memory() for h in hx]
     hy = [torch.empty(PREFILL_M, lin["N"], dtype=torch.float16).pin_memory() for lin in layer]
 
+    # Three streams: the upload of linear i + 1 and the download of linear i - 1 run beside the GEMM of linear i (PCIe is full
+    # duplex).  A step starts after the one before it has finished on all three, and ends when its last download has.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
     def e2e_step():
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        s_in.wait_event(start)
+        s_out.wait_event(start)
         for lin, H, X, Y, HY in zip(layer, hx, xs, ys, hy):
-            X.copy_(H, non_blocking=True)
+            with torch.cuda.stream(s_in):
+                X.copy_(H, non_blocking=True)
+                up = torch.cuda.Event()
+                up.record(s_in)
+            cur.wait_event(up)
             b.esp_spgemm(X, lin["packed"], lin["perm"], Y, po, pws)
-            HY.copy_(Y, non_blocking=True)
+            done = torch.cuda.Event()
+            done.record(cur)
+            s_out.wait_event(done)
+            with torch.cuda.stream(s_out):
+                HY.copy_(Y, non_blocking=True)
+        last = torch.cuda.Event()
+        last.record(s_out)
+        cur.wait_event(last)
     e2e_ms = time_steps(e2e_step, max(2, args.steps // 4), 2)
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     e2e = {"value": whole_job_rate(flops, world, e2e_ms) / 1e12, "unit": "TFLOP/s",
@@ -407,7 +427,18 @@ def run_ours(args):
         fbytes = sum(gemm_bytes(DECODE_M, N, K) for N, K in fused)
         extra["decode_fused_qkv_gateup"] = {"launches_per_layer": 4, "ms_per_step": fms, "value": fbytes / (fms * 1e-3) / 1e9,
                                             "unit": "GB/s", "frac_of_measured_hbm": fbytes / (fms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-        del fpk, fx, fy
+        # the same fused layer at prefill size (four tiling passes and four GEMMs per step)
+        fpx = [torch.randn(K, PREFILL_M, device=dev).half() for _, K in fused]
+        fpy = [torch.empty(PREFILL_M, N, dtype=torch.float16, device=dev) for N, _ in fused]
+        fpws = torch.empty(max(b.esp_spgemm_workspace_bytes(PREFILL_M, N, K, fo) for N, K in fused), dtype=torch.uint8, device=dev)
+
+        def fused_prefill_step():
+            for pk, pm, X, Y in zip(fpk, fperm, fpx, fpy):
+                b.esp_spgemm(X, pk, pm, Y, fo, fpws)
+        fpms = graph_time(fused_prefill_step, 4)
+        extra["prefill_fused_qkv_gateup"] = {"calls_per_layer": 4, "ms_per_step": fpms, "value": flops / (fpms * 1e-3) / 1e12,
+                                             "unit": "TFLOP/s"}
+        del fpk, fx, fy, fpx, fpy, fpws
         # ---------------- dense cuBLAS fp16 on the same shapes (library call, context) ----------------
         def dense_step(xs_):
             for lin, X in zip(layer, xs_):

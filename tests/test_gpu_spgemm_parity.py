@@ -266,7 +266,12 @@ def test_llama7b_shapes_sampled_outputs():
         for M in (1, 16, 128, 2048):
             X = inputs.make_gemm_x(wl, lin, M)
             Y = spgemm(X, packed, theta, N)
-            rows = np.unique(np.concatenate([g.choice(M, min(M, 8), replace=False), [0, M - 1, min(M - 1, 255), min(M - 1, 256)]]))
-            cols = np.unique(np.concatenate([g.choice(N, 48, replace=False), [0, 127, 128, N - 1]]))
+            edges = [0, M - 1] + [min(M - 1, e) for e in (119, 120, 223, 224, 239, 240, 255, 256)]   # token-tile seams
+            rows = np.unique(np.concatenate([g.choice(M, min(M, 8), replace=False), edges]))
+            cols = np.unique(np.concatenate([g.choice(N, 48, replace=False), [0, 127, 128, 511, 512, N - 1]]))
             Yref = orc.product_entries(X, vals, meta, theta, rows, cols)
             check(Y[np.ix_(rows, cols)], Yref)
+            if M == 2048:       # the configuration bench.py times: channel-major X, static weights, full workspace
+                Yc = spgemm(X, packed, theta, N, channel_major=True, static_weights=1)
+                check(Yc[np.ix_(rows, cols)], Yref)
+                assert np.array_equal(Yc, Y)        # both layouts feed the same MMAs in the same order
