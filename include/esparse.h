@@ -165,6 +165,7 @@ enum { ESP_X_TOKEN_MAJOR = 0,    /* X[t, c] at X + t * ldx + c  (tokens are rows
        ESP_X_CHANNEL_MAJOR = 1 };/* X[t, c] at X + c * ldx + t  (channels are rows: the activation
                                     handed over transposed)                                           */
 enum { ESP_OUT_F16 = 0, ESP_OUT_F32 = 1 };
+enum { ESP_ACT_NONE = 0, ESP_ACT_RELU = 1 };
 enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_GATHER = 1,    /* element gather of X, any layout, no workspace (slow for large M)    */
        ESP_KERNEL_TMA = 2,       /* channel-major X rows fetched four at a time by the tensor memory
@@ -192,6 +193,11 @@ typedef struct {
                                     a programmatic dependent of the preceding kernel: its weight prefetch
                                     overlaps that kernel's tail, and only the reads of X and the writes
                                     of Y wait for it.  0 (default) = plain stream order.                 */
+    int activation;              /* ESP_ACT_*: applied to the fp32 sum (+ bias) before it is rounded to
+                                    the output type.  The paper times the bare product (Table 5); OPT's
+                                    linears carry a bias and fc1 a ReLU, which this folds into the same
+                                    launch                                                               */
+    const void *bias;            /* device fp16 [N], added to every token row; NULL = none            */
 } esp_gemm_opts;
 
 void esp_gemm_opts_default(esp_gemm_opts *opts);

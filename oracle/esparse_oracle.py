@@ -346,6 +346,20 @@ def product_entries(X: np.ndarray, vals: np.ndarray, meta: np.ndarray, theta: Op
     return product(np.asarray(X)[rows], np.asarray(vals)[cols], np.asarray(meta)[cols], theta)
 
 
+def layer_output(Y: np.ndarray, bias: Optional[np.ndarray] = None, relu: bool = False) -> np.ndarray:
+    """What a linear layer hands on: the product plus a per-feature bias (the same for every token), then ReLU.
+    The paper times the bare product (Table 5); OPT's linears carry a bias and its first feed-forward linear a ReLU."""
+    out = np.asarray(Y, dtype=np.float64).copy()
+    if bias is not None:
+        b = np.asarray(bias).astype(np.float64)
+        assert b.shape == (out.shape[1],)
+        for t in range(out.shape[0]):
+            out[t, :] = out[t, :] + b
+    if relu:
+        out[out < 0.0] = 0.0
+    return out
+
+
 # ----------------------------------------------------------------------------- whole producer
 @dataclass
 class PruneResult:

@@ -18,6 +18,7 @@ ESP_ERR_STATIC_LIMIT = 8
 ESP_STATIC_SCRATCH_BYTES = 8 << 20
 ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
+ESP_ACT_NONE, ESP_ACT_RELU = 0, 1
 ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR, ESP_KERNEL_PAIR_TILED = 0, 1, 2, 4, 5, 6
 
 
@@ -35,7 +36,8 @@ class esp_prune_stats(ctypes.Structure):
 
 class esp_gemm_opts(ctypes.Structure):
     _fields_ = [("struct_size", c_size_t), ("x_layout", c_int), ("out_dtype", c_int), ("split_k", c_int),
-                ("force_kernel", c_int), ("token_tile", c_int), ("static_weights", c_int)]
+                ("force_kernel", c_int), ("token_tile", c_int), ("static_weights", c_int), ("activation", c_int),
+                ("bias", c_void_p)]
 
 
 class EsparseError(RuntimeError):

@@ -47,6 +47,8 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
         o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR && o->force_kernel != ESP_KERNEL_PAIR_TILED)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
+    if (o->activation != ESP_ACT_NONE && o->activation != ESP_ACT_RELU) return ESP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(o->bias) & 1u) != 0) return ESP_ERR_ALIGNMENT;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
 }
@@ -100,6 +102,8 @@ void esp_gemm_opts_default(esp_gemm_opts *o) {
     o->force_kernel = ESP_KERNEL_AUTO;
     o->token_tile = 0;
     o->static_weights = 0;
+    o->activation = ESP_ACT_NONE;
+    o->bias = nullptr;
 }
 
 size_t esp_metric_prune_workspace_bytes(int No, int C, int T, const esp_prune_opts *opts) {

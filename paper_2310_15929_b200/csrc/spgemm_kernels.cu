@@ -37,7 +37,22 @@ struct GemmParams {
     int k_tiles_per_split;
     const uint8_t *ximg;     // tiled pair kernel: permuted X as shared-memory images (written by xtile_kernel)
     const uint32_t *xflags;  // one word per image: 1 once it is complete
+    const __half *bias;      // [N] added to every token row before the activation, or NULL
+    int act;                 // ESP_ACT_*
 };
+
+// Bias and activation on the finished fp32 sum of one output element (never on a K-slice's partial sum).
+__device__ __forceinline__ float epilogue_value(const GemmParams &p, float acc, long feature) {
+    if (p.bias != nullptr && feature < p.N) {
+        // volatile: the fp16 overload of __ldg is a plain (non-volatile) asm statement, which the compiler may execute
+        // ahead of the null test above; with bias == NULL that read address 2 * feature and faulted
+        unsigned short h;
+        asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(h) : "l"(p.bias + feature) : "memory");
+        acc += __half2float(__ushort_as_half(h));
+    }
+    if (p.act == ESP_ACT_RELU) acc = fmaxf(acc, 0.f);
+    return acc;
+}
 
 // ---------------------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -319,8 +334,9 @@ __global__ void __launch_bounds__(192) spgemm_gather_kernel(const GemmParams p) 
                     for (int e = 0; e < 16; ++e) {
                         const int t = tok0 + c0 + e;
                         if (t < p.M) {
-                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
-                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
+                            const float y = epilogue_value(p, __uint_as_float(v[e]), feature);
+                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = y;
+                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(y);
                         }
                     }
                 }
@@ -346,6 +362,7 @@ __global__ void __launch_bounds__(192) spgemm_gather_kernel(const GemmParams p) 
             float acc = 0.f;
             for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
             if (ok) {
+                acc = epilogue_value(p, acc, feature);
                 if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
                 else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
             }
@@ -518,8 +535,9 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
                     for (int e = 0; e < 16; ++e) {
                         const int t = tok0 + c0 + e;
                         if (t < p.M) {
-                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = __uint_as_float(v[e]);
-                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(__uint_as_float(v[e]));
+                            const float y = epilogue_value(p, __uint_as_float(v[e]), feature);
+                            if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = y;
+                            else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(y);
                         }
                     }
                 }
@@ -544,6 +562,7 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
             float acc = 0.f;
             for (int r = 0; r < split; ++r) acc += ld_dsmem_f32(sbase + (uint32_t)idx * 4u, (uint32_t)r);
             if (ok) {
+                acc = epilogue_value(p, acc, feature);
                 if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = acc;
                 else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(acc);
             }
@@ -877,12 +896,16 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
 #pragma unroll
                     for (int e = 0; e < 16; ++e) v[e] = 0;
                 }
+                const long feature = (long)ft * 128 + f_local;
                 if (p.out_f32) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
+                    for (int e = 0; e < 16; ++e)
+                        reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = epilogue_value(p, __uint_as_float(v[e]), feature);
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
+                    for (int e = 0; e < 16; ++e)
+                        reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] =
+                            __float2half_rn(epilogue_value(p, __uint_as_float(v[e]), feature));
                 }
             }
             tc_fence_before();
@@ -965,6 +988,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
                 float acc = 0.f;
                 for (int r = 0; r < split; ++r) acc += recv[(r * 128 + f) * cnt + i];   // slice order: deterministic
                 const long o = (long)t * p.ldy + (long)ft * 128 + f;
+                acc = epilogue_value(p, acc, (long)ft * 128 + f);
                 if (p.out_f32) reinterpret_cast<float *>(p.Y)[o] = acc;
                 else reinterpret_cast<__half *>(p.Y)[o] = __float2half_rn(acc);
             }
@@ -992,8 +1016,9 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
                 const long o = (long)t * p.ldy + (long)ft * 128 + f0;
                 for (int e = 0; e < 4; ++e)
                     if (f0 + e < f_valid) {
-                        if (p.out_f32) reinterpret_cast<float *>(p.Y)[o + e] = a[e];
-                        else reinterpret_cast<__half *>(p.Y)[o + e] = __float2half_rn(a[e]);
+                        const float y = epilogue_value(p, a[e], (long)ft * 128 + f0 + e);
+                        if (p.out_f32) reinterpret_cast<float *>(p.Y)[o + e] = y;
+                        else reinterpret_cast<__half *>(p.Y)[o + e] = __float2half_rn(y);
                     }
             }
         }
@@ -1342,6 +1367,8 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.perm = perm;
     p.Y = Y; p.ldy = ldy;
     p.out_f32 = (o.out_dtype == ESP_OUT_F32) ? 1 : 0;
+    p.bias = reinterpret_cast<const __half *>(o.bias);
+    p.act = o.activation;
     p.k_tiles = ceil_div(K, kTileK);
     p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
     p.ximg = nullptr;

@@ -549,8 +549,9 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 }
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    if (sizeof(OutT) == 4) reinterpret_cast<float *>(area)[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
-                    else reinterpret_cast<__half *>(area)[(c0 + e) * 128 + f_local] = __float2half_rn(__uint_as_float(v[e]));
+                    const float y = epilogue_value(p, __uint_as_float(v[e]), (long)ftile[a] * 128 + f_local);
+                    if (sizeof(OutT) == 4) reinterpret_cast<float *>(area)[(c0 + e) * 128 + f_local] = y;
+                    else reinterpret_cast<__half *>(area)[(c0 + e) * 128 + f_local] = __float2half_rn(y);
                 }
             }
         };

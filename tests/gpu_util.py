@@ -60,7 +60,7 @@ def pack_on_gpu(vals, meta):
 
 
 def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0, token_tile=0, kernel=0,
-           workspace=True, static_weights=0):
+           workspace=True, static_weights=0, bias=None, relu=False):
     dev = torch.device(DEV)
     M = X.shape[0]
     Xd = torch.from_numpy(np.ascontiguousarray(X)).to(dev)
@@ -75,6 +75,11 @@ def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0
     o.out_dtype = b.ESP_OUT_F32 if out_f32 else b.ESP_OUT_F16
     o.split_k, o.token_tile, o.force_kernel = split_k, token_tile, kernel
     o.static_weights = static_weights
+    bias_d = None
+    if bias is not None:
+        bias_d = torch.from_numpy(np.ascontiguousarray(bias, dtype=np.float16)).to(dev)
+        o.bias = bias_d.data_ptr()
+    o.activation = b.ESP_ACT_RELU if relu else b.ESP_ACT_NONE
     Y = torch.full((M, N), float("nan"), dtype=torch.float32 if out_f32 else torch.float16, device=dev)
     th = None if theta is None else torch.from_numpy(np.ascontiguousarray(theta, dtype=np.int32)).to(dev)
     ws = None

@@ -275,3 +275,28 @@ def test_llama7b_shapes_sampled_outputs():
                 Yc = spgemm(X, packed, theta, N, channel_major=True, static_weights=1)
                 check(Yc[np.ix_(rows, cols)], Yref)
                 assert np.array_equal(Yc, Y)        # both layouts feed the same MMAs in the same order
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 200, 264), (130, 384, 1160), (520, 640, 1160)])
+def test_bias_and_relu_epilogue(M, N, K):
+    """Bias (per feature) and ReLU applied to the finished fp32 sum in every kernel's epilogue, K-sliced launches
+    included (where a partial sum must not see them), against the oracle's product + bias -> ReLU."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(M + N, N, K)
+    g = np.random.default_rng(M)
+    X = g.standard_normal((M, K)).astype(np.float16)
+    bias = (g.standard_normal(N) * 2).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Y0 = orc.product(X, vals, meta, theta)
+    variants = [dict(kernel=1, workspace=False), dict(kernel=1, channel_major=True, split_k=2), dict(kernel=4, channel_major=True),
+                dict(kernel=4, channel_major=True, split_k=2), dict(kernel=4, channel_major=True, split_k=3),
+                dict(kernel=4, channel_major=True, token_tile=128, split_k=2), dict(kernel=2, channel_major=True, token_tile=64), dict()]
+    if M > 256:
+        variants += [dict(kernel=5, channel_major=True), dict(kernel=6, channel_major=True), dict(kernel=6)]
+    for kw in variants:
+        for relu in (False, True):
+            ref = orc.layer_output(Y0, bias, relu)
+            check(spgemm(X, packed, theta, N, bias=bias, relu=relu, **kw), ref)
+            check(spgemm(X, packed, theta, N, bias=bias, relu=relu, out_f32=True, **kw), ref, True)
+    relu_only = spgemm(X, packed, theta, N, relu=True)
+    assert (relu_only >= 0).all() and (relu_only == 0).any()

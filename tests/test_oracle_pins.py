@@ -461,3 +461,16 @@ def test_metric_prune_config0_end_to_end_properties():
     kept = orc.decompress_permuted(np.ones_like(r.vals), r.meta) != 0
     xi = orc.metric(W, r.score)[:, r.theta]
     assert abs(xi[kept].sum() - r.obj_after_lbs) <= 1e-11 * r.obj_after_lbs
+
+
+def test_layer_output_bias_runs_along_features_and_relu_clamps():
+    """Pins of the epilogue: a worked example (bias per feature, not per token), zero bias and no ReLU is the identity,
+    ReLU output is non-negative and leaves positive entries untouched."""
+    Y = np.array([[1.0, -2.0, 3.0], [-4.0, 5.0, -6.0]])            # 2 tokens x 3 features
+    bias = np.array([10.0, 0.5, -1.0], dtype=np.float16)
+    assert np.array_equal(orc.layer_output(Y, bias), np.array([[11.0, -1.5, 2.0], [6.0, 5.5, -7.0]]))
+    assert np.array_equal(orc.layer_output(Y, bias, relu=True), np.array([[11.0, 0.0, 2.0], [6.0, 5.5, 0.0]]))
+    assert np.array_equal(orc.layer_output(Y), Y)
+    assert np.array_equal(orc.layer_output(Y, np.zeros(3, np.float16)), Y)
+    with pytest.raises(AssertionError):
+        orc.layer_output(Y, np.zeros(2, np.float16))                # a bias per token is refused
