@@ -213,6 +213,19 @@ void esp_gemm_opts_default(esp_gemm_opts *opts);
 size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts);
 
 /*
+ * The search of step (2) of "Efficient Sparse-GEMM Implementation" (the paper tries the library's algorithms per weight
+ * shape and keeps the fastest): times esp_spgemm on the caller's buffers for every (kernel, token tile, K-slices) the
+ * sizes admit, `reps` calls each after one untimed call, the configuration in *opts first, and writes the fastest into
+ * opts->force_kernel / token_tile / split_k (the other fields are kept).  best_us / planned_us (optional, host) receive
+ * the time per call of the winner and of the configuration *opts came in with.  Y and the workspace are written; the
+ * stream is synchronised.  Persisting the three integers per (M, N, K, layout) is the caller's: binding.py has
+ * save_plan_table / load_plan_table.
+ */
+esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
+                             void *Y, long ldy, esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, int reps,
+                             float *best_us, float *planned_us, void *cuda_stream);
+
+/*
  * Reports the launch configuration esp_spgemm would use for these sizes on the current device (the
  * counterpart of step (2) of "Efficient Sparse-GEMM Implementation", where the paper searches the library's
  * algorithms per weight shape): kernel (ESP_KERNEL_*), tokens per CTA tile, K-slices per cluster, pipeline

@@ -55,7 +55,7 @@ EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_ge
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
            "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout", "esp_calib_state_bytes", "esp_calib_reset",
-           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish")
+           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish", "esp_spgemm_tune")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -205,6 +205,55 @@ def esp_spgemm(X, packed, perm, Y, opts, workspace=None, stream=None):
                         0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream))
     if st != ESP_OK:
         raise EsparseError(st, "esp_spgemm")
+
+
+_lib.esp_spgemm_tune.restype = c_int
+_lib.esp_spgemm_tune.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
+                                 POINTER(esp_gemm_opts), c_void_p, c_size_t, c_int, POINTER(ctypes.c_float),
+                                 POINTER(ctypes.c_float), c_void_p]
+
+
+def esp_spgemm_tune(X, packed, perm, Y, opts, workspace=None, reps=5, stream=None) -> dict:
+    """Times the admissible launch configurations on these buffers and writes the fastest into `opts` (see the header).
+    Returns {"kernel", "token_tile", "split_k", "best_us", "planned_us"}."""
+    M, N = Y.shape
+    K = X.shape[0] if opts.x_layout == ESP_X_CHANNEL_MAJOR else X.shape[1]
+    best, planned = ctypes.c_float(), ctypes.c_float()
+    st = int(_lib.esp_spgemm_tune(_ptr(X), M, K, X.stride(0), _ptr(packed), _ptr(perm), N, _ptr(Y), Y.stride(0),
+                                  ctypes.byref(opts), _ptr(workspace),
+                                  0 if workspace is None else workspace.numel() * workspace.element_size(), reps,
+                                  ctypes.byref(best), ctypes.byref(planned), _stream(stream)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_spgemm_tune")
+    return {"kernel": opts.force_kernel, "token_tile": opts.token_tile, "split_k": opts.split_k,
+            "best_us": best.value, "planned_us": planned.value}
+
+
+def plan_key(M: int, N: int, K: int, opts: esp_gemm_opts) -> str:
+    return f"{M}x{N}x{K}:layout{opts.x_layout}:out{opts.out_dtype}:static{opts.static_weights}"
+
+
+def save_plan_table(path: str, table: dict) -> None:
+    """Persists tuned configurations: {plan_key(...): {"kernel": .., "token_tile": .., "split_k": ..}} as JSON."""
+    import json
+    with open(path, "w") as f:
+        json.dump({k: {"kernel": int(v["kernel"]), "token_tile": int(v["token_tile"]), "split_k": int(v["split_k"])}
+                   for k, v in table.items()}, f, indent=1, sort_keys=True)
+
+
+def load_plan_table(path: str) -> dict:
+    import json
+    with open(path) as f:
+        return json.load(f)
+
+
+def apply_plan(opts: esp_gemm_opts, table: dict, M: int, N: int, K: int) -> bool:
+    """Sets opts.force_kernel / token_tile / split_k from the table's entry for these sizes; False if there is none."""
+    e = table.get(plan_key(M, N, K, opts))
+    if e is None:
+        return False
+    opts.force_kernel, opts.token_tile, opts.split_k = e["kernel"], e["token_tile"], e["split_k"]
+    return True
 
 
 def esp_spgemm_static_raw(X, M, K, ldx, packed, perm, N, Y, ldy, out_dtype, stream) -> int:

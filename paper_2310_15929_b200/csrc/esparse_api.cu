@@ -2,6 +2,7 @@
 #include "esp_common.cuh"
 
 #include <mutex>
+#include <vector>
 
 namespace esp {
 
@@ -255,6 +256,77 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packe
     if (st != ESP_OK) return st;
     return launch_spgemm((const __half *)X, M, K, ldx, packed, perm, N, Y, ldy, *opts, plan, workspace,
                          workspace_bytes, (cudaStream_t)cuda_stream);
+}
+
+esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
+                             void *Y, long ldy, esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, int reps,
+                             float *best_us, float *planned_us, void *cuda_stream) {
+    esp_status_t st = check_gemm_opts(opts);
+    if (st != ESP_OK) return st;
+    if (reps < 1 || reps > 1000) return ESP_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return ESP_ERR_CUDA;
+    }
+    // candidates: the planner's own choice first, then every (kernel, token tile, K-slices) the sizes admit
+    struct Cand { int kernel, tile, split; };
+    std::vector<Cand> cands;
+    cands.push_back({opts->force_kernel, opts->token_tile, opts->split_k});
+    if (M > 256) {
+        for (int tile : {240, 224, 192, 128}) {
+            cands.push_back({ESP_KERNEL_PAIR_TILED, tile, 1});
+            cands.push_back({ESP_KERNEL_PAIR, tile, 1});
+        }
+        cands.push_back({ESP_KERNEL_PAIR, 256, 1});
+    }
+    if (M <= 1024) {
+        for (int tile : {16, 32, 64, 128, 256}) {
+            if (tile < M && tile < 256 && (M + tile - 1) / tile > 8) continue;      // many narrow token tiles: never the best
+            if (tile >= 2 * M && tile > 16) continue;
+            for (int split = 1; split <= 8; ++split) cands.push_back({ESP_KERNEL_STREAM, tile, split});
+        }
+    }
+    esp_gemm_opts best = *opts;
+    float best_t = -1.f, first_t = -1.f;
+    esp_status_t result = ESP_OK;
+    for (size_t i = 0; i < cands.size(); ++i) {
+        esp_gemm_opts o = *opts;
+        o.force_kernel = cands[i].kernel;
+        o.token_tile = cands[i].tile;
+        o.split_k = cands[i].split;
+        GemmPlan plan;
+        const bool have_ws = workspace && aligned16(workspace);
+        if (check_gemm_opts(&o) != ESP_OK || plan_gemm(M, N, K, o, have_ws ? workspace_bytes : 0, &plan) != ESP_OK) continue;
+        if (i > 0 && plan.split_k != cands[i].split && cands[i].kernel == ESP_KERNEL_STREAM) continue;   // stepped down: a duplicate
+        // one untimed call (first-use set-up, caches), then `reps` timed ones
+        st = esp_spgemm(X, M, K, ldx, packed, perm, N, Y, ldy, &o, workspace, workspace_bytes, cuda_stream);
+        if (st != ESP_OK) {
+            if (i == 0) { result = st; break; }        // the caller's own configuration must work
+            continue;
+        }
+        cudaEventRecord(e0, stream);
+        for (int r = 0; r < reps && st == ESP_OK; ++r)
+            st = esp_spgemm(X, M, K, ldx, packed, perm, N, Y, ldy, &o, workspace, workspace_bytes, cuda_stream);
+        cudaEventRecord(e1, stream);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { result = ESP_ERR_CUDA; break; }
+        if (st != ESP_OK) continue;
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const float us = ms * 1000.f / (float)reps;
+        if (i == 0) first_t = us;
+        if (best_t < 0.f || us < best_t) { best_t = us; best = o; }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (result != ESP_OK) return result;
+    if (best_t < 0.f) return ESP_ERR_UNSUPPORTED;
+    if (esp_last_device_status() != ESP_OK) return ESP_ERR_TIMEOUT;
+    *opts = best;
+    if (best_us) *best_us = best_t;
+    if (planned_us) *planned_us = first_t;
+    return ESP_OK;
 }
 
 esp_status_t esp_selftest_wait_timeout(void *cuda_stream) {

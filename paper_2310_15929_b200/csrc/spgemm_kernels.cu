@@ -41,17 +41,25 @@ struct GemmParams {
     int act;                 // ESP_ACT_*
 };
 
-// Bias and activation on the finished fp32 sum of one output element (never on a K-slice's partial sum).
-__device__ __forceinline__ float epilogue_value(const GemmParams &p, float acc, long feature) {
+// Bias and activation on the finished fp32 sum of one output element (never on a K-slice's partial sum).  The bias of a
+// feature is fetched once per thread (epilogue_bias) and applied to all of that feature's tokens (epilogue_apply).
+__device__ __forceinline__ float epilogue_bias(const GemmParams &p, long feature) {
+    float b = 0.f;
     if (p.bias != nullptr && feature < p.N) {
         // volatile: the fp16 overload of __ldg is a plain (non-volatile) asm statement, which the compiler may execute
         // ahead of the null test above; with bias == NULL that read address 2 * feature and faulted
         unsigned short h;
-        asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(h) : "l"(p.bias + feature) : "memory");
-        acc += __half2float(__ushort_as_half(h));
+        asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(h) : "l"(p.bias + feature));
+        b = __half2float(__ushort_as_half(h));
     }
-    if (p.act == ESP_ACT_RELU) acc = fmaxf(acc, 0.f);
-    return acc;
+    return b;
+}
+__device__ __forceinline__ float epilogue_apply(float acc, float bias, int act) {
+    acc += bias;
+    return act == ESP_ACT_RELU ? fmaxf(acc, 0.f) : acc;
+}
+__device__ __forceinline__ float epilogue_value(const GemmParams &p, float acc, long feature) {
+    return epilogue_apply(acc, epilogue_bias(p, feature), p.act);
 }
 
 // ---------------------------------------------------------------------------------------------- PTX helpers
@@ -319,6 +327,7 @@ __global__ void __launch_bounds__(192) spgemm_gather_kernel(const GemmParams p) 
         bool ok = alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
         tc_fence_after();
         float *stage_f32 = reinterpret_cast<float *>(smem);
+        const float bias_f = epilogue_bias(p, feature);
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 16) {
             uint32_t v[16];
@@ -334,7 +343,7 @@ __global__ void __launch_bounds__(192) spgemm_gather_kernel(const GemmParams p) 
                     for (int e = 0; e < 16; ++e) {
                         const int t = tok0 + c0 + e;
                         if (t < p.M) {
-                            const float y = epilogue_value(p, __uint_as_float(v[e]), feature);
+                            const float y = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
                             if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = y;
                             else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(y);
                         }
@@ -520,6 +529,7 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
         const bool ok = (nk == 0 || mbar_wait(accum_bar, 0, abort_flag));
         tc_fence_after();
         float *stage_f32 = reinterpret_cast<float *>(smem);
+        const float bias_f = epilogue_bias(p, feature);
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 16) {
             uint32_t v[16];
@@ -535,7 +545,7 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
                     for (int e = 0; e < 16; ++e) {
                         const int t = tok0 + c0 + e;
                         if (t < p.M) {
-                            const float y = epilogue_value(p, __uint_as_float(v[e]), feature);
+                            const float y = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
                             if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = y;
                             else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(y);
                         }
@@ -887,6 +897,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
         if (split == 1) {
             // accumulators -> shared memory [token][128 features] in the output type -> 16-byte stores
             const int esize = p.out_f32 ? 4 : 2;
+            const float bias_f = epilogue_bias(p, (long)ft * 128 + f_local);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 uint32_t v[16];
@@ -896,16 +907,15 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
 #pragma unroll
                     for (int e = 0; e < 16; ++e) v[e] = 0;
                 }
-                const long feature = (long)ft * 128 + f_local;
                 if (p.out_f32) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e)
-                        reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = epilogue_value(p, __uint_as_float(v[e]), feature);
+                        reinterpret_cast<float *>(smem)[(c0 + e) * 128 + f_local] = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
                 } else {
 #pragma unroll
                     for (int e = 0; e < 16; ++e)
                         reinterpret_cast<__half *>(smem)[(c0 + e) * 128 + f_local] =
-                            __float2half_rn(epilogue_value(p, __uint_as_float(v[e]), feature));
+                            __float2half_rn(epilogue_apply(__uint_as_float(v[e]), bias_f, p.act));
                 }
             }
             tc_fence_before();

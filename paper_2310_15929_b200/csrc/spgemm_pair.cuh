@@ -538,6 +538,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         // fp16 output: both accumulators are staged side by side (2 x TN x 256 bytes) and stored in one sweep.
         auto stage_acc = [&](int a, uint8_t *area, auto out_tag) {
             using OutT = decltype(out_tag);
+            const float bias_f = epilogue_bias(p, (long)ftile[a] * 128 + f_local);
 #pragma unroll 1
             for (int c0 = cgrp * 16; c0 < TN; c0 += 64) {
                 uint32_t v[16];
@@ -549,7 +550,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 }
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float y = epilogue_value(p, __uint_as_float(v[e]), (long)ftile[a] * 128 + f_local);
+                    const float y = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
                     if (sizeof(OutT) == 4) reinterpret_cast<float *>(area)[(c0 + e) * 128 + f_local] = y;
                     else reinterpret_cast<__half *>(area)[(c0 + e) * 128 + f_local] = __float2half_rn(y);
                 }

@@ -141,3 +141,18 @@ def test_calibration_state_size_and_argument_checks():
     assert b.esp_calib_state_bytes(C, 1) == 0
     assert b._lib.esp_calib_reset(None, C, bins, None) == b.ESP_ERR_INVALID_ARG
     assert b._lib.esp_calib_range(None, None, 4, C, C, bins, None) == b.ESP_ERR_INVALID_ARG
+
+
+def test_plan_table_round_trip(tmp_path):
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    table = {b.plan_key(16, 4096, 4096, o): {"kernel": b.ESP_KERNEL_STREAM, "token_tile": 16, "split_k": 8}}
+    path = str(tmp_path / "plans.json")
+    b.save_plan_table(path, table)
+    loaded = b.load_plan_table(path)
+    assert loaded == table
+    assert b.apply_plan(o, loaded, 16, 4096, 4096)
+    assert (o.force_kernel, o.token_tile, o.split_k) == (b.ESP_KERNEL_STREAM, 16, 8)
+    assert not b.apply_plan(o, loaded, 17, 4096, 4096)
+    o2 = b.esp_gemm_opts_default()                       # another layout is another entry
+    assert not b.apply_plan(o2, loaded, 16, 4096, 4096)

@@ -300,3 +300,33 @@ def test_bias_and_relu_epilogue(M, N, K):
             check(spgemm(X, packed, theta, N, bias=bias, relu=relu, out_f32=True, **kw), ref, True)
     relu_only = spgemm(X, packed, theta, N, relu=True)
     assert (relu_only >= 0).all() and (relu_only == 0).any()
+
+
+@pytest.mark.parametrize("M,N,K,channel_major", [(16, 512, 1024, True), (520, 640, 1160, False)])
+def test_tuned_configuration_is_valid_and_no_slower_than_the_plan(M, N, K, channel_major):
+    """esp_spgemm_tune tries every admissible (kernel, token tile, K-slices), returns the fastest; that configuration
+    must reproduce the oracle's product, and its time cannot exceed the planner's own (which is the first candidate)."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    vals, meta, theta = pruned(M + K, N, K)
+    X = np.random.default_rng(M).standard_normal((M, K)).astype(np.float16)
+    dev = torch.device("cuda:0")
+    packed = pack_on_gpu(vals, meta)
+    Xd = torch.from_numpy(X).to(dev)
+    if channel_major:
+        Xd = Xd.t().contiguous()
+    th = torch.from_numpy(theta).to(dev)
+    Y = torch.empty(M, N, dtype=torch.float16, device=dev)
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR if channel_major else b.ESP_X_TOKEN_MAJOR
+    nws = b.esp_spgemm_workspace_bytes(M, N, K, o)
+    ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+    r = b.esp_spgemm_tune(Xd, packed, th, Y, o, ws, reps=3)
+    assert r["best_us"] > 0 and r["best_us"] <= r["planned_us"]
+    assert (o.force_kernel, o.token_tile, o.split_k) == (r["kernel"], r["token_tile"], r["split_k"])
+    Y.fill_(float("nan"))
+    b.esp_spgemm(Xd, packed, th, Y, o, ws)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    check(Y.cpu().numpy(), orc.product(X, vals, meta, theta))
