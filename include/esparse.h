@@ -69,6 +69,9 @@ typedef struct {
     int use_gns;                 /* 0 skips the global naive shuffle (identity start order)           */
     int use_lbs;                 /* 0 skips the local block shuffle                                   */
     const double *score_override;/* optional device f64[C]: use these s_c instead of computing them   */
+    int global_bin_range;        /* Eq. 1 does not say what is divided into K bins.  0 (default): each channel's
+                                    own [min, max]; 1: the layer's [min, max] over all channels, so that a
+                                    narrow channel falls into few bins and gets a low entropy             */
     const int32_t *perm_override;/* optional device i32[C]: start from this channel order instead of the
                                     global shuffle's (a stored permutation, e.g. to re-compress updated
                                     weights); the block shuffle still runs on it if use_lbs is set.

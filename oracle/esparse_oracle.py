@@ -90,8 +90,11 @@ def channel_norm(xcal: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------- O2 entropy
-def channel_histogram(xcal: np.ndarray, bins: int = BINS) -> np.ndarray:
+def channel_histogram(xcal: np.ndarray, bins: int = BINS, global_range: bool = False) -> np.ndarray:
     """Counts n[c,k] of Eq. 1's bins.
+
+    global_range=True is the other reading of "divide it into K bins": one range [lo, hi] for the whole layer
+    (minimum and maximum over all channels) instead of each channel's own.
 
     Reading: the K bins are equal-width on the channel's own range [lo_c, hi_c],
     left-closed, the maximum falls in the last bin; raw signed values are binned.
@@ -107,6 +110,9 @@ def channel_histogram(xcal: np.ndarray, bins: int = BINS) -> np.ndarray:
         w = x.shape[1]
         lo = x.min(axis=0)
         hi = x.max(axis=0)
+        if global_range:
+            lo = np.full(w, float(xcal.min()))
+            hi = np.full(w, float(xcal.max()))
         rng = hi - lo
         safe = np.where(rng > 0, rng, 1.0)
         idx = np.floor(((x - lo[None, :]) * float(bins)) / safe[None, :])
@@ -129,9 +135,9 @@ def entropy_from_counts(counts: np.ndarray, T: int) -> np.ndarray:
     return ir
 
 
-def channel_entropy(xcal: np.ndarray, bins: int = BINS) -> np.ndarray:
+def channel_entropy(xcal: np.ndarray, bins: int = BINS, global_range: bool = False) -> np.ndarray:
     x = np.asarray(xcal)
-    return entropy_from_counts(channel_histogram(x, bins), x.shape[0])
+    return entropy_from_counts(channel_histogram(x, bins, global_range), x.shape[0])
 
 
 # ----------------------------------------------------------------------------- O3 score / metric
@@ -382,12 +388,12 @@ class PruneResult:
 def metric_prune(W: np.ndarray, xcal: np.ndarray, alpha: float, *, bins: int = BINS,
                  use_entropy: bool = True, use_norm: bool = True, use_gns: bool = True, use_lbs: bool = True,
                  lbs_block: int = LBS_BLOCK, lbs_max_swaps: int = 0, score: Optional[np.ndarray] = None,
-                 objectives: bool = True) -> PruneResult:
+                 objectives: bool = True, global_bin_range: bool = False) -> PruneResult:
     """norm -> entropy -> score -> global shuffle -> block shuffle -> 2:4 selection -> compression."""
     W = np.asarray(W, dtype=np.float16)
     C = W.shape[1]
     am = channel_norm(xcal)
-    ir = channel_entropy(xcal, bins)
+    ir = channel_entropy(xcal, bins, global_bin_range)
     s = channel_score(ir, am, alpha, use_entropy, use_norm) if score is None else np.asarray(score, np.float64)
     mean = channel_mean_metric(W, s)
     ident = np.arange(C, dtype=np.int32)

@@ -26,7 +26,7 @@ class esp_prune_opts(ctypes.Structure):
     _fields_ = [("struct_size", c_size_t), ("alpha", c_double), ("bins", c_int), ("n_keep", c_int),
                 ("m_group", c_int), ("lbs_block", c_int), ("lbs_max_swaps", c_int), ("use_entropy", c_int),
                 ("use_norm", c_int), ("use_gns", c_int), ("use_lbs", c_int), ("score_override", c_void_p),
-                ("perm_override", c_void_p)]
+                ("global_bin_range", c_int), ("perm_override", c_void_p)]
 
 
 class esp_prune_stats(ctypes.Structure):

@@ -36,6 +36,7 @@ static esp_status_t check_prune_opts(const esp_prune_opts *o) {
     if (o->bins < 2 || o->bins > 512) return ESP_ERR_UNSUPPORTED;
     if (o->lbs_block < 4 || o->lbs_block > 256 || o->lbs_block % 4 != 0) return ESP_ERR_INVALID_ARG;
     if (o->lbs_max_swaps < 0) return ESP_ERR_INVALID_ARG;
+    if (o->global_bin_range != 0 && o->global_bin_range != 1) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
 }
 
@@ -91,6 +92,7 @@ void esp_prune_opts_default(esp_prune_opts *o) {
     o->use_gns = 1;
     o->use_lbs = 1;
     o->score_override = nullptr;
+    o->global_bin_range = 0;
     o->perm_override = nullptr;
 }
 

@@ -93,6 +93,23 @@ __global__ void colstats_finish_kernel(int C, int splits, const double *__restri
     hi[c] = (double)mx;
 }
 
+// The layer-wide bin range: every channel's [lo, hi] replaced by the minimum and maximum over all channels (one CTA).
+__global__ void __launch_bounds__(1024) global_range_kernel(int C, double *__restrict__ lo, double *__restrict__ hi) {
+    __shared__ double s_lo[32], s_hi[32];
+    double mn = INFINITY, mx = -INFINITY;
+    for (int c = threadIdx.x; c < C; c += 1024) { mn = fmin(mn, lo[c]); mx = fmax(mx, hi[c]); }
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fmin(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        mx = fmax(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    }
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = mn; s_hi[threadIdx.x >> 5] = mx; }
+    __syncthreads();
+    mn = s_lo[0]; mx = s_hi[0];
+    for (int w = 1; w < 32; ++w) { mn = fmin(mn, s_lo[w]); mx = fmax(mx, s_hi[w]); }
+    __syncthreads();
+    for (int c = threadIdx.x; c < C; c += 1024) { lo[c] = mn; hi[c] = mx; }
+}
+
 // Streaming calibration: fold one chunk's partial statistics into the running state (chunk order = call order).
 __global__ void calib_merge_kernel(int C, int splits, const double *__restrict__ part_sumsq, const float *__restrict__ part_min,
                                    const float *__restrict__ part_max, double *__restrict__ sumsq, double *__restrict__ lo,
@@ -949,6 +966,7 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
                                                                              w.part_min, w.part_max);
         colstats_finish_kernel<<<cblocks, cthreads, 0, stream>>>(C, w.splits, w.part_sumsq, w.part_min, w.part_max,
                                                                  w.norm, w.lo, w.hi);
+        if (o.global_bin_range) global_range_kernel<<<1, 1024, 0, stream>>>(C, w.lo, w.hi);
         // K2
         ESP_CUDA_OK(cudaMemsetAsync(w.counts, 0, sizeof(unsigned int) * (size_t)C * o.bins, stream));
         const int hsplits = pick_splits(T, ceil_div(C, 64), di.sm_count);

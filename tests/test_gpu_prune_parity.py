@@ -221,3 +221,22 @@ def test_streaming_calibration_equals_one_shot(C, splits):
     assert np.array_equal(perm, ref.theta) or ref.near_tie_sort > 0
     if np.array_equal(perm, ref.theta):
         assert_masks_match(vals, meta, ref)
+
+
+@pytest.mark.parametrize("No,C,T", [(128, 264, 333), (96, 1024, 200)])
+def test_global_bin_range_variant(No, C, T):
+    """Layer-wide bin range (the other reading of Eq. 1): entropy and score to the statistics bar, masks bit-exact given
+    the oracle's own near-tie count, and different from the per-channel reading on this input."""
+    from tests.gpu_util import GpuPrune
+    W, X = layer(300 + C, No, C, T)
+    X[:, 9] = (X[:, 9].astype(np.float32) / 64).astype(np.float16)          # a narrow channel
+    alpha = 1.0 / math.sqrt(T)
+    g = GpuPrune(W, X, alpha, use_lbs=0, global_bin_range=1)
+    ir = orc.channel_entropy(X, global_range=True)
+    assert np.allclose(g.entropy.cpu().numpy(), ir, rtol=STAT_RTOL, atol=1e-14)
+    assert ir[9] < 0.5 * orc.channel_entropy(X)[9]
+    ref = orc.metric_prune(W, X, alpha, use_lbs=False, global_bin_range=True, objectives=False)
+    vals, meta, perm = g.host()
+    assert np.array_equal(perm, ref.theta) or ref.near_tie_sort > 0
+    if np.array_equal(perm, ref.theta):
+        assert_masks_match(vals, meta, ref)

@@ -474,3 +474,26 @@ def test_layer_output_bias_runs_along_features_and_relu_clamps():
     assert np.array_equal(orc.layer_output(Y, np.zeros(3, np.float16)), Y)
     with pytest.raises(AssertionError):
         orc.layer_output(Y, np.zeros(2, np.float16))                # a bias per token is refused
+
+
+def test_global_bin_range_reading_of_eq1():
+    """The other reading of Eq. 1's bins (one range for the layer): a channel spread over the whole range keeps ln K, a
+    channel that is narrow against the layer collapses into one bin (entropy 0) although its own-range entropy is
+    ln 4; identical channels give the same counts under both readings; counts still sum to T."""
+    T = 100
+    wide = np.arange(100, dtype=np.float64)                          # 0..99, one value per bin of [0, 99]
+    narrow = np.repeat([0.0, 0.25, 0.5, 0.75], 25)
+    X = np.stack([wide, narrow], axis=1).astype(np.float16)
+    per = orc.channel_entropy(X)
+    glob = orc.channel_entropy(X, global_range=True)
+    assert abs(per[0] - math.log(100)) < 1e-12 and abs(glob[0] - math.log(100)) < 1e-12
+    assert abs(per[1] - math.log(4)) < 1e-12
+    assert glob[1] == 0.0
+    counts = orc.channel_histogram(X, global_range=True)
+    assert counts.sum(axis=1).tolist() == [T, T] and counts[1, 0] == T
+    same = np.stack([wide, wide[::-1]], axis=1).astype(np.float16)   # same value set in both channels
+    assert np.array_equal(orc.channel_histogram(same), orc.channel_histogram(same, global_range=True))
+    # the own-range reading is blind to a channel's scale, the layer-range reading is not
+    X2 = X.copy(); X2[:, 1] *= 64                                     # exact in fp16
+    assert np.allclose(orc.channel_entropy(X2)[1], per[1], rtol=0, atol=1e-12)
+    assert orc.channel_entropy(X2, global_range=True)[1] > 1.0
