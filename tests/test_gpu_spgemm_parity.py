@@ -330,3 +330,55 @@ def test_tuned_configuration_is_valid_and_no_slower_than_the_plan(M, N, K, chann
     torch.cuda.synchronize()
     assert b.esp_last_device_status() == b.ESP_OK
     check(Y.cpu().numpy(), orc.product(X, vals, meta, theta))
+
+
+def test_prefill_calls_replayed_from_a_cuda_graph_share_one_workspace():
+    """What bench.py times: several large-M calls recorded once into a CUDA graph, all using one workspace (X images and
+    their flags are rewritten by every call), replayed with new inputs.  Every replay must give the product of the inputs it
+    ran on: a flag left up by the previous call or replay must never let a GEMM read an image early."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    dev = torch.device("cuda:0")
+    M = 520
+    shapes = [(640, 1160), (384, 512), (256, 1160)]
+    g = np.random.default_rng(21)
+    layers = []
+    for N, K in shapes:
+        vals, meta, theta = pruned(N + K, N, K)
+        layers.append(dict(N=N, K=K, vals=vals, meta=meta, theta=theta, packed=pack_on_gpu(vals, meta),
+                           th=torch.from_numpy(theta).to(dev), X=torch.empty(K, M, dtype=torch.float16, device=dev),
+                           Y=torch.empty(M, N, dtype=torch.float16, device=dev)))
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    o.static_weights = 1
+    ws = torch.empty(max(b.esp_spgemm_workspace_bytes(M, L["N"], L["K"], o) for L in layers), dtype=torch.uint8, device=dev)
+    ws.fill_(0xFF)                                            # flags start as garbage
+
+    def run_all(stream):
+        for L in layers:
+            b.esp_spgemm(L["X"], L["packed"], L["th"], L["Y"], o, ws, stream=stream)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    for L in layers:
+        L["X"].copy_(torch.from_numpy(g.standard_normal((L["K"], M)).astype(np.float16)))
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        run_all(side)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            run_all(side)
+    torch.cuda.synchronize()
+    for replay in range(3):
+        host_x = []
+        for L in layers:
+            x = g.standard_normal((L["K"], M)).astype(np.float16)
+            host_x.append(x)
+            L["X"].copy_(torch.from_numpy(x))
+            L["Y"].fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert b.esp_last_device_status() == b.ESP_OK
+        for L, x in zip(layers, host_x):
+            check(L["Y"].cpu().numpy(), orc.product(np.ascontiguousarray(x.T), L["vals"], L["meta"], L["theta"]))
