@@ -412,7 +412,7 @@ def run_ours(args):
                            "launch": "CUDA graph of 20 layer passes, static_weights=1",
                            "plain_stream_order_gbs": dbytes / (dms_plain * 1e-3) / 1e9,
                            "tuned_gbs": dbytes / (dms_tuned * 1e-3) / 1e9,
-                           "tuned_configs": [[t.force_kernel, t.token_tile, t.split_k] for t in tuned],
+                           "tuned_configs": [[t.force_kernel, t.token_tile, t.split_k, t.pipeline_stages] for t in tuned],
                            "roofline": {"bound": "hbm", "achieved": dgbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                         "frac": dgbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES,
                                         "frac_of_nominal_8TBs": dgbs / 8000.0, "of": peaks["source"]}}

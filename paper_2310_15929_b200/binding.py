@@ -36,7 +36,7 @@ class esp_prune_stats(ctypes.Structure):
 
 class esp_gemm_opts(ctypes.Structure):
     _fields_ = [("struct_size", c_size_t), ("x_layout", c_int), ("out_dtype", c_int), ("split_k", c_int),
-                ("force_kernel", c_int), ("token_tile", c_int), ("static_weights", c_int), ("activation", c_int),
+                ("force_kernel", c_int), ("token_tile", c_int), ("static_weights", c_int), ("pipeline_stages", c_int), ("activation", c_int),
                 ("bias", c_void_p)]
 
 
@@ -226,7 +226,7 @@ def esp_spgemm_tune(X, packed, perm, Y, opts, workspace=None, reps=5, stream=Non
     if st != ESP_OK:
         raise EsparseError(st, "esp_spgemm_tune")
     return {"kernel": opts.force_kernel, "token_tile": opts.token_tile, "split_k": opts.split_k,
-            "best_us": best.value, "planned_us": planned.value}
+            "pipeline_stages": opts.pipeline_stages, "best_us": best.value, "planned_us": planned.value}
 
 
 def plan_key(M: int, N: int, K: int, opts: esp_gemm_opts) -> str:
@@ -237,7 +237,8 @@ def save_plan_table(path: str, table: dict) -> None:
     """Persists tuned configurations: {plan_key(...): {"kernel": .., "token_tile": .., "split_k": ..}} as JSON."""
     import json
     with open(path, "w") as f:
-        json.dump({k: {"kernel": int(v["kernel"]), "token_tile": int(v["token_tile"]), "split_k": int(v["split_k"])}
+        json.dump({k: {"kernel": int(v["kernel"]), "token_tile": int(v["token_tile"]), "split_k": int(v["split_k"]),
+                       "pipeline_stages": int(v.get("pipeline_stages", 0))}
                    for k, v in table.items()}, f, indent=1, sort_keys=True)
 
 
@@ -253,6 +254,7 @@ def apply_plan(opts: esp_gemm_opts, table: dict, M: int, N: int, K: int) -> bool
     if e is None:
         return False
     opts.force_kernel, opts.token_tile, opts.split_k = e["kernel"], e["token_tile"], e["split_k"]
+    opts.pipeline_stages = e.get("pipeline_stages", 0)
     return True
 
 

@@ -50,6 +50,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->activation != ESP_ACT_NONE && o->activation != ESP_ACT_RELU) return ESP_ERR_INVALID_ARG;
+    if (o->pipeline_stages != 0 && (o->pipeline_stages < 2 || o->pipeline_stages > 12)) return ESP_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(o->bias) & 1u) != 0) return ESP_ERR_ALIGNMENT;
     if (o->token_tile < 0 || o->token_tile > 256 || o->token_tile % 16 != 0) return ESP_ERR_INVALID_ARG;
     return ESP_OK;
@@ -105,6 +106,7 @@ void esp_gemm_opts_default(esp_gemm_opts *o) {
     o->force_kernel = ESP_KERNEL_AUTO;
     o->token_tile = 0;
     o->static_weights = 0;
+    o->pipeline_stages = 0;
     o->activation = ESP_ACT_NONE;
     o->bias = nullptr;
 }
@@ -273,21 +275,22 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
         return ESP_ERR_CUDA;
     }
     // candidates: the planner's own choice first, then every (kernel, token tile, K-slices) the sizes admit
-    struct Cand { int kernel, tile, split; };
+    struct Cand { int kernel, tile, split, stages; };
     std::vector<Cand> cands;
-    cands.push_back({opts->force_kernel, opts->token_tile, opts->split_k});
+    cands.push_back({opts->force_kernel, opts->token_tile, opts->split_k, opts->pipeline_stages});
     if (M > 256) {
         for (int tile : {240, 224, 192, 128}) {
-            cands.push_back({ESP_KERNEL_PAIR_TILED, tile, 1});
-            cands.push_back({ESP_KERNEL_PAIR, tile, 1});
+            cands.push_back({ESP_KERNEL_PAIR_TILED, tile, 1, 0});
+            cands.push_back({ESP_KERNEL_PAIR, tile, 1, 0});
         }
-        cands.push_back({ESP_KERNEL_PAIR, 256, 1});
+        cands.push_back({ESP_KERNEL_PAIR, 256, 1, 0});
     }
     if (M <= 1024) {
         for (int tile : {16, 32, 64, 128, 256}) {
             if (tile < M && tile < 256 && (M + tile - 1) / tile > 8) continue;      // many narrow token tiles: never the best
             if (tile >= 2 * M && tile > 16) continue;
-            for (int split = 1; split <= 8; ++split) cands.push_back({ESP_KERNEL_STREAM, tile, split});
+            for (int split = 1; split <= 8; ++split)
+                for (int stages : {0, 2, 3, 4, 6, 8}) cands.push_back({ESP_KERNEL_STREAM, tile, split, stages});
         }
     }
     esp_gemm_opts best = *opts;
@@ -298,10 +301,13 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
         o.force_kernel = cands[i].kernel;
         o.token_tile = cands[i].tile;
         o.split_k = cands[i].split;
+        o.pipeline_stages = cands[i].stages;
         GemmPlan plan;
         const bool have_ws = workspace && aligned16(workspace);
         if (check_gemm_opts(&o) != ESP_OK || plan_gemm(M, N, K, o, have_ws ? workspace_bytes : 0, &plan) != ESP_OK) continue;
-        if (i > 0 && plan.split_k != cands[i].split && cands[i].kernel == ESP_KERNEL_STREAM) continue;   // stepped down: a duplicate
+        if (i > 0 && cands[i].kernel == ESP_KERNEL_STREAM &&
+            (plan.split_k != cands[i].split || (cands[i].stages != 0 && plan.stages != cands[i].stages)))
+            continue;                                                          // stepped down or clamped: a duplicate
         // one untimed call (first-use set-up, caches), then `reps` timed ones
         st = esp_spgemm(X, M, K, ldx, packed, perm, N, Y, ldy, &o, workspace, workspace_bytes, cuda_stream);
         if (st != ESP_OK) {

@@ -1329,6 +1329,10 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 const size_t budget = (size_t)di.max_smem_optin / r - (r > 1 ? 1024 : 0);
                 if (budget < fixed + 2 * per_stage) break;
                 int stages = (int)((budget - fixed) / per_stage);
+                if (o.pipeline_stages > 0) {                              // a requested ring depth: this one only, if it fits
+                    if (r > 1 || fixed + (size_t)o.pipeline_stages * per_stage > (size_t)di.max_smem_optin) break;
+                    stages = o.pipeline_stages;
+                }
                 if (stages > kMaxStages) stages = kMaxStages;
                 if (stages > kts) stages = kts < 2 ? 2 : kts;
                 if (stages == last_stages) continue;
@@ -1341,7 +1345,9 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 const bool pow2 = (split & (split - 1)) == 0;
                 double cost = (double)waves * (kts + 2.0) + (split > 1 ? (pow2 ? 0.25 : 6.0) + 0.05 * split : 0.0) + 0.01 * r;
                 // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
-                if (o.static_weights && 2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin) cost += 3.0;
+                if (o.static_weights && o.pipeline_stages == 0 &&
+                    2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin)
+                    cost += 3.0;
                 if (getenv("ESP_LOG"))
                     fprintf(stderr, "esparse plan M=%d N=%d K=%d tile=%d: split=%d stages=%d capacity=%d ctas=%ld waves=%ld cost=%.2f\n", M, N, K,
                             bn, split, stages, cap, ctas, waves, cost);
