@@ -220,11 +220,12 @@ size_t esp_spgemm_workspace_bytes(int M, int N, int K, const esp_gemm_opts *opts
 /*
  * The search of step (2) of "Efficient Sparse-GEMM Implementation" (the paper tries the library's algorithms per weight
  * shape and keeps the fastest): times esp_spgemm on the caller's buffers for every (kernel, token tile, K-slices) the
- * sizes admit, `reps` calls each after one untimed call, the configuration in *opts first, and writes the fastest into
- * opts->force_kernel / token_tile / split_k (the other fields are kept).  best_us / planned_us (optional, host) receive
- * the time per call of the winner and of the configuration *opts came in with.  Y and the workspace are written; the
- * stream is synchronised.  Persisting the three integers per (M, N, K, layout) is the caller's: binding.py has
- * save_plan_table / load_plan_table.
+ * sizes admit (and every ring depth of the streaming kernel), `reps` calls each after one untimed call, the configuration
+ * in *opts first, and writes the fastest into opts->force_kernel / token_tile / split_k / pipeline_stages (the other
+ * fields are kept).  best_us / planned_us (optional, host) receive the time per call of the winner and of the
+ * configuration *opts came in with.  The calls repeat on the same buffers, so small weights are timed from L2.  Y and the
+ * workspace are written; the stream is synchronised.  Persisting the four integers per (M, N, K, layout) is the
+ * caller's: binding.py has save_plan_table / load_plan_table.
  */
 esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
                              void *Y, long ldy, esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, int reps,
@@ -246,7 +247,10 @@ esp_status_t esp_spgemm_plan(int M, int N, int K, const esp_gemm_opts *opts, int
  *   X       fp16, M tokens x K channels in the layout opts->x_layout names, leading dimension ldx
  *           (elements; multiple of 8)
  *   packed  esp_packed_bytes(N, K) bytes from esp_metric_prune / esp_pack
- *   perm    int32 [K] or NULL for the identity; fused into the X-tile load, X is never copied
+ *   perm    int32 [K] or NULL for the identity; applied while the X tile is loaded (up to 256 tokens, or without
+ *           a workspace) or by the pass that writes the X operand images into the workspace (more tokens)
+ *   opts    layout, output type, optional bias and activation: Y = act(product + bias), bias and activation applied
+ *           to the finished fp32 sum
  *   Y       out, [M, N] row-major (Y[t, j] at Y + t * ldy + j), fp16 or fp32 per opts->out_dtype
  *
  * The result does not depend on scheduling: K-slices are summed in slice order.
