@@ -1283,13 +1283,16 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
     }
     if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED) {
         if (bn == 0) {
-            // widest token tile unless a narrower one saves a whole wave of clusters: cost ~ waves x tile width
+            // cost ~ waves of clusters x time of one channel step: the longer of the step's MMAs (8 x TN/2 clocks) and its
+            // 36 KB of weights + X tile (64-token blocks: 16 KB for TN = 128, else 32 KB) at the ~70 B/clk an SM pulls from
+            // L2.  Wide tiles win once the grid fills the machine; a grid of less than one wave runs faster on narrow ones.
             const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
-            long best = -1;
-            for (int tn : {240, 224, 192}) {
+            double best = -1.0;
+            for (int tn : {240, 224, 192, 128}) {
                 const long clusters = f_pairs * ceil_div(M, tn);
-                const long cost = ceil_div(clusters, per_wave) * tn;
-                if (best < 0 || cost < best) { best = cost; bn = tn; }
+                const double mma = 4.0 * tn, copy = (36864.0 + (tn > 128 ? 32768.0 : 16384.0)) / 70.0;
+                const double cost = (double)ceil_div(clusters, per_wave) * (mma > copy ? mma : copy) * (k_tiles + 12.0);
+                if (best < 0.0 || cost < best) { best = cost; bn = tn; }
             }
         }
         if (bn != 128 && bn != 192 && bn != 224 && bn != 240 && bn != 256) return ESP_ERR_INVALID_ARG;
@@ -1343,9 +1346,13 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 const long waves = (ctas + cap - 1) / cap;
                 // (2, 4 or 8 slices push their partial rows as vectors; other counts go element by element: measured ~2 us slower)
                 const bool pow2 = (split & (split - 1)) == 0;
-                double cost = (double)waves * (kts + 2.0) + (split > 1 ? (pow2 ? 0.25 : 6.0) + 0.05 * split : 0.0) + 0.01 * r;
+                // per CTA: kts steps + set-up, reduction and epilogue, which grow with the token tile (measured: a 256-token
+                // tile in one wave of 32 steps beats three waves of 8)
+                double cost = (double)waves * (kts + 2.0 + bn / 32.0) + (split > 1 ? (pow2 ? 0.25 : 6.0) + 0.05 * split : 0.0) + 0.01 * r;
                 // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
-                if (o.static_weights && o.pipeline_stages == 0 &&
+                // (not when every CTA has an SM of its own anyway: a deeper ring is then free, measured 16.0 -> 12.6 us on
+                // 4096 x 4096 at 64 tokens)
+                if (o.static_weights && o.pipeline_stages == 0 && ctas > di.sm_count &&
                     2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin)
                     cost += 3.0;
                 if (getenv("ESP_LOG"))
