@@ -197,7 +197,8 @@ typedef struct {
                                     overlaps that kernel's tail, and only the reads of X and the writes
                                     of Y wait for it.  0 (default) = plain stream order.                 */
     int pipeline_stages;         /* depth of the streaming kernel's shared-memory ring (2..12 tiles in flight
-                                    per CTA); 0 = choose.  Ignored by the other kernels.               */
+                                    per CTA; clamped to what shared memory holds and to the channel steps of
+                                    a K-slice); 0 = choose.  Ignored by the other kernels.              */
     int activation;              /* ESP_ACT_*: applied to the fp32 sum (+ bias) before it is rounded to
                                     the output type.  The paper times the bare product (Table 5); OPT's
                                     linears carry a bias and fc1 a ReLU, which this folds into the same

@@ -1332,9 +1332,9 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 const size_t budget = (size_t)di.max_smem_optin / r - (r > 1 ? 1024 : 0);
                 if (budget < fixed + 2 * per_stage) break;
                 int stages = (int)((budget - fixed) / per_stage);
-                if (o.pipeline_stages > 0) {                              // a requested ring depth: this one only, if it fits
-                    if (r > 1 || fixed + (size_t)o.pipeline_stages * per_stage > (size_t)di.max_smem_optin) break;
-                    stages = o.pipeline_stages;
+                if (o.pipeline_stages > 0) {                              // a requested ring depth: this one only, or what fits
+                    if (r > 1) break;
+                    if (stages > o.pipeline_stages) stages = o.pipeline_stages;
                 }
                 if (stages > kMaxStages) stages = kMaxStages;
                 if (stages > kts) stages = kts < 2 ? 2 : kts;

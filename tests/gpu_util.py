@@ -60,7 +60,7 @@ def pack_on_gpu(vals, meta):
 
 
 def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0, token_tile=0, kernel=0,
-           workspace=True, static_weights=0, bias=None, relu=False):
+           workspace=True, static_weights=0, bias=None, relu=False, pipeline_stages=0):
     dev = torch.device(DEV)
     M = X.shape[0]
     Xd = torch.from_numpy(np.ascontiguousarray(X)).to(dev)
@@ -75,6 +75,7 @@ def spgemm(X, packed, theta, N, *, channel_major=False, out_f32=False, split_k=0
     o.out_dtype = b.ESP_OUT_F32 if out_f32 else b.ESP_OUT_F16
     o.split_k, o.token_tile, o.force_kernel = split_k, token_tile, kernel
     o.static_weights = static_weights
+    o.pipeline_stages = pipeline_stages
     bias_d = None
     if bias is not None:
         bias_d = torch.from_numpy(np.ascontiguousarray(bias, dtype=np.float16)).to(dev)

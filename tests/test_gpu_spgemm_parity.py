@@ -382,3 +382,23 @@ def test_prefill_calls_replayed_from_a_cuda_graph_share_one_workspace():
         assert b.esp_last_device_status() == b.ESP_OK
         for L, x in zip(layers, host_x):
             check(L["Y"].cpu().numpy(), orc.product(np.ascontiguousarray(x.T), L["vals"], L["meta"], L["theta"]))
+
+
+@pytest.mark.parametrize("M,K", [(16, 2048), (130, 1160)])
+def test_requested_ring_depth_of_the_streaming_kernel(M, K):
+    """Every ring depth the option admits (clamped to the channel steps of a K-slice) gives the same product, bit for
+    bit: the depth changes when tiles are loaded, not what is summed in which order."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    N = 384
+    vals, meta, theta = pruned(K + M, N, K)
+    X = np.random.default_rng(K).standard_normal((M, K)).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Yref = orc.product(X, vals, meta, theta)
+    base = spgemm(X, packed, theta, N, channel_major=True, kernel=4, split_k=2, out_f32=True)
+    check(base, Yref, True)
+    for stages in (2, 3, 4, 6, 12):
+        y = spgemm(X, packed, theta, N, channel_major=True, kernel=4, split_k=2, out_f32=True, pipeline_stages=stages)
+        assert np.array_equal(y, base), stages
+    from paper_2310_15929_b200 import binding as b
+    with pytest.raises(b.EsparseError):
+        spgemm(X, packed, theta, N, channel_major=True, kernel=4, pipeline_stages=1)
