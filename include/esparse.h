@@ -262,6 +262,20 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx,
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Several independent products in one launch: Y[i] = X[i] . P[i] . W_s[i]^T for i < count <= ESP_MAX_GROUP, each with its
+ * own weight, permutation, input and output.  (The paper times a layer's Q/K/V as one GEMM, Table 5; this keeps the three
+ * weights, and their three channel permutations, separate.)  M, K, ldx and the options are common, N[i] and ldy[i] are
+ * per problem; X, packed, perm, N, Y, ldy are HOST arrays of `count` entries (perm[i] may be NULL; opts->bias is not
+ * supported here and must be NULL).  Up to 256 tokens the problems share one launch of the streaming kernel -- what a
+ * short launch loses to start-up and drain is paid once; for more tokens the call is the same as `count` calls of
+ * esp_spgemm.  workspace: count * esp_spgemm_workspace_bytes(M, max N, K, opts) bytes.
+ */
+#define ESP_MAX_GROUP 4
+esp_status_t esp_spgemm_grouped(int count, const void *const *X, int M, int K, long ldx, const void *const *packed,
+                                const int32_t *const *perm, const int *N, void *const *Y, const long *ldy,
+                                const esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The product for hosts that cannot allocate device memory.  (The paper has no counterpart: this is a
  * deployment convenience of this library, not a step of the method.)
  *

@@ -55,7 +55,7 @@ EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_ge
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
            "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout", "esp_calib_state_bytes", "esp_calib_reset",
-           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish", "esp_spgemm_tune")
+           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish", "esp_spgemm_tune", "esp_spgemm_grouped")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -227,6 +227,27 @@ def esp_spgemm_tune(X, packed, perm, Y, opts, workspace=None, reps=5, stream=Non
         raise EsparseError(st, "esp_spgemm_tune")
     return {"kernel": opts.force_kernel, "token_tile": opts.token_tile, "split_k": opts.split_k,
             "pipeline_stages": opts.pipeline_stages, "best_us": best.value, "planned_us": planned.value}
+
+
+_lib.esp_spgemm_grouped.restype = c_int
+_lib.esp_spgemm_grouped.argtypes = [c_int, POINTER(c_void_p), c_int, c_int, c_long, POINTER(c_void_p), POINTER(c_void_p),
+                                    POINTER(c_int), POINTER(c_void_p), POINTER(c_long), POINTER(esp_gemm_opts), c_void_p,
+                                    c_size_t, c_void_p]
+
+
+def esp_spgemm_grouped(Xs, packeds, perms, Ys, opts, workspace=None, stream=None):
+    """Ys[i] = Xs[i] . P[i] . W_s[i]^T for up to 4 problems with common M and K in one call (one launch up to 256 tokens)."""
+    n = len(Ys)
+    M = Ys[0].shape[0]
+    K = Xs[0].shape[0] if opts.x_layout == ESP_X_CHANNEL_MAJOR else Xs[0].shape[1]
+    arr = lambda items: (c_void_p * n)(*[_ptr(t) for t in items])
+    Ns = (c_int * n)(*[y.shape[1] for y in Ys])
+    ldys = (c_long * n)(*[y.stride(0) for y in Ys])
+    st = int(_lib.esp_spgemm_grouped(n, arr(Xs), M, K, Xs[0].stride(0), arr(packeds), arr(perms), Ns, arr(Ys), ldys,
+                                     ctypes.byref(opts), _ptr(workspace),
+                                     0 if workspace is None else workspace.numel() * workspace.element_size(), _stream(stream)))
+    if st != ESP_OK:
+        raise EsparseError(st, "esp_spgemm_grouped")
 
 
 def plan_key(M: int, N: int, K: int, opts: esp_gemm_opts) -> str:

@@ -88,6 +88,10 @@ struct GemmPlan {
 esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan);
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o);        // everything any plan could use
 size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o);    // below this only the gather kernel runs
+// One streaming-kernel launch for `count` problems; ESP_ERR_UNSUPPORTED if these sizes do not plan onto that kernel.
+esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, long ldx, const void *const *packed,
+                                 const int32_t *const *perm, const int *N, void *const *Y, const long *ldy,
+                                 const esp_gemm_opts &o, void *workspace, size_t workspace_bytes, cudaStream_t stream);
 esp_status_t launch_wait_timeout_selftest(cudaStream_t stream);
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm,
                            int N, void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan,

@@ -262,6 +262,38 @@ esp_status_t esp_spgemm(const void *X, int M, int K, long ldx, const void *packe
                          workspace_bytes, (cudaStream_t)cuda_stream);
 }
 
+esp_status_t esp_spgemm_grouped(int count, const void *const *X, int M, int K, long ldx, const void *const *packed,
+                                const int32_t *const *perm, const int *N, void *const *Y, const long *ldy,
+                                const esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    esp_status_t st = check_gemm_opts(opts);
+    if (st != ESP_OK) return st;
+    if (count < 1 || count > ESP_MAX_GROUP || !X || !packed || !N || !Y || !ldy || opts->bias) return ESP_ERR_INVALID_ARG;
+    if (M <= 0 || K <= 0 || K % 8 != 0) return ESP_ERR_SHAPE;
+    if (opts->x_layout == ESP_X_TOKEN_MAJOR ? (ldx < K) : (ldx < M)) return ESP_ERR_SHAPE;
+    if (ldx % 8 != 0) return ESP_ERR_ALIGNMENT;
+    for (int i = 0; i < count; ++i) {
+        if (!X[i] || !packed[i] || !Y[i]) return ESP_ERR_INVALID_ARG;
+        if (N[i] <= 0 || ldy[i] < N[i]) return ESP_ERR_SHAPE;
+        if (!aligned16(X[i]) || !aligned16(packed[i]) || !aligned16(Y[i]) || (perm && !aligned16(perm[i]))) return ESP_ERR_ALIGNMENT;
+    }
+    DeviceInfo di;
+    st = device_info(&di);
+    if (st != ESP_OK) return st;
+    if (di.cc_major != 10) return ESP_ERR_UNSUPPORTED;
+    const bool have_ws = workspace && aligned16(workspace);
+    st = launch_spgemm_group(count, X, M, K, ldx, packed, perm, N, Y, ldy, *opts, have_ws ? workspace : nullptr,
+                             have_ws ? workspace_bytes : 0, (cudaStream_t)cuda_stream);
+    if (st != ESP_ERR_UNSUPPORTED) return st;
+    // sizes that do not plan onto one streaming launch: the problems one after the other, each with its share of the workspace
+    const size_t share = have_ws ? (workspace_bytes / (size_t)count) & ~(size_t)255 : 0;
+    for (int i = 0; i < count; ++i) {
+        st = esp_spgemm(X[i], M, K, ldx, packed[i], perm ? perm[i] : nullptr, N[i], Y[i], ldy[i], opts,
+                        share ? (uint8_t *)workspace + (size_t)i * share : nullptr, share, cuda_stream);
+        if (st != ESP_OK) return st;
+    }
+    return ESP_OK;
+}
+
 esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,
                              void *Y, long ldy, esp_gemm_opts *opts, void *workspace, size_t workspace_bytes, int reps,
                              float *best_us, float *planned_us, void *cuda_stream) {

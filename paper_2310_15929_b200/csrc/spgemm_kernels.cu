@@ -41,6 +41,14 @@ struct GemmParams {
     int act;                 // ESP_ACT_*
 };
 
+// Up to ESP_MAX_GROUP independent products in one launch of the streaming kernel: the feature tiles of the problems
+// follow each other along grid.x (problem i owns tiles [ft_start[i], ft_start[i + 1])); M, K and the launch shape are common.
+struct GemmGroup {
+    int count;
+    int ft_start[ESP_MAX_GROUP + 1];
+    GemmParams p[ESP_MAX_GROUP];
+};
+
 // Bias and activation on the finished fp32 sum of one output element (never on a K-slice's partial sum).  The bias of a
 // feature is fetched once per thread (epilogue_bias) and applied to all of that feature's tokens (epilogue_apply).
 __device__ __forceinline__ float epilogue_bias(const GemmParams &p, long feature) {
@@ -730,8 +738,14 @@ __device__ __forceinline__ void push_columns_pow2(const uint32_t (&v)[16], int c
 }
 
 template <int BN>
-__global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(const GemmParams p, const int stages) {
+__global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(const GemmGroup grp, const int stages) {
     using L = StreamCfg<BN>;
+    // this CTA's problem: selected with constant indices so that the parameters stay in registers
+    GemmParams p = grp.p[0];
+    int ft_first = 0;
+#pragma unroll
+    for (int i = 1; i < ESP_MAX_GROUP; ++i)
+        if (i < grp.count && (int)blockIdx.x >= grp.ft_start[i]) { p = grp.p[i]; ft_first = grp.ft_start[i]; }
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -750,7 +764,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     int *perm_s = reinterpret_cast<int *>(smem + perm_off);          // [kPermRing][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ft = blockIdx.x, tok0 = blockIdx.y * BN;
+    const int ft = (int)blockIdx.x - ft_first, tok0 = blockIdx.y * BN;
     const int kt_begin = slice * p.k_tiles_per_split;
     const int kt_end = min(p.k_tiles, kt_begin + p.k_tiles_per_split);
     const int nk = max(0, kt_end - kt_begin);
@@ -1061,7 +1075,35 @@ esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int sp
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 2 : 1;
-    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, stages));
+    GemmGroup grp;
+    grp.count = 1;
+    for (int i = 0; i <= ESP_MAX_GROUP; ++i) grp.ft_start[i] = i == 0 ? 0 : f_tiles;
+    for (int i = 0; i < ESP_MAX_GROUP; ++i) grp.p[i] = p;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, grp, stages));
+    return ESP_OK;
+}
+
+// The same launch for a group of problems (feature tiles concatenated along grid.x).
+template <int BN>
+esp_status_t launch_stream_group(const GemmGroup &grp, int t_tiles, int split, int stages, bool dependent, cudaStream_t stream) {
+    auto kern = spgemm_stream_kernel<BN>;
+    const size_t smem = stream_smem_bytes(BN, stages, split);
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grp.ft_start[grp.count], t_tiles, split);
+    cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = split;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, grp, stages));
     return ESP_OK;
 }
 
@@ -1475,6 +1517,63 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
         case 64: return launch_gather<64, 5>(p, f_tiles, t_tiles, plan.split_k, stream);
         case 128: return launch_gather<128, 4>(p, f_tiles, t_tiles, plan.split_k, stream);
         case 256: return launch_gather<256, 2>(p, f_tiles, t_tiles, plan.split_k, stream);
+        default: return ESP_ERR_INVALID_ARG;
+    }
+}
+
+esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, long ldx, const void *const *packed,
+                                 const int32_t *const *perm, const int *N, void *const *Y, const long *ldy,
+                                 const esp_gemm_opts &o, void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (M > 256) return ESP_ERR_UNSUPPORTED;
+    int f_total = 0;
+    for (int i = 0; i < count; ++i) f_total += ceil_div(N[i], kTileFeat);
+    const size_t tbytes = transpose_bytes(M, K, o);
+    if (tbytes > 0 && (!workspace || workspace_bytes < tbytes * (size_t)count)) return ESP_ERR_UNSUPPORTED;
+    GemmPlan plan;
+    esp_status_t st = plan_gemm(M, f_total * kTileFeat, K, o, workspace ? workspace_bytes : 0, &plan);
+    if (st != ESP_OK) return st;
+    if (plan.kernel != ESP_KERNEL_STREAM) return ESP_ERR_UNSUPPORTED;
+    GemmGroup grp;
+    grp.count = count;
+    int ft = 0;
+    for (int i = 0; i < ESP_MAX_GROUP; ++i) {
+        const int j = i < count ? i : 0;
+        GemmParams &p = grp.p[i];
+        p.X = (const __half *)X[j]; p.ldx = ldx; p.M = M; p.K = K; p.N = N[j];
+        p.x_channel_major = 1;
+        p.packed = (const uint8_t *)packed[j];
+        p.perm = perm ? perm[j] : nullptr;
+        p.Y = Y[j]; p.ldy = ldy[j];
+        p.out_f32 = (o.out_dtype == ESP_OUT_F32) ? 1 : 0;
+        p.bias = nullptr;
+        p.act = o.activation;
+        p.k_tiles = ceil_div(K, kTileK);
+        p.k_tiles_per_split = ceil_div(p.k_tiles, plan.split_k);
+        p.ximg = nullptr;
+        p.xflags = nullptr;
+        grp.ft_start[i] = ft;
+        if (i < count) {
+            if (o.x_layout != ESP_X_CHANNEL_MAJOR) {      // token-major: a transposed copy per problem, one after the other
+                const long ldt = transposed_ld(M);
+                uint16_t *xt = reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(workspace) + (size_t)i * tbytes);
+                transpose_x_kernel<<<dim3(ceil_div(K, 32), ceil_div(ldt, 32)), 256, 0, stream>>>(
+                    reinterpret_cast<const uint16_t *>(X[i]), M, K, ldx, xt, ldt);
+                ESP_CUDA_OK(cudaGetLastError());
+                p.X = reinterpret_cast<const __half *>(xt);
+                p.ldx = ldt;
+            }
+            ft += ceil_div(N[i], kTileFeat);
+        }
+    }
+    for (int i = count; i <= ESP_MAX_GROUP; ++i) grp.ft_start[i] = ft;
+    const int t_tiles = ceil_div(M, plan.token_tile);
+    const bool dependent = o.static_weights != 0;
+    switch (plan.token_tile) {
+        case 16: return launch_stream_group<16>(grp, t_tiles, plan.split_k, plan.stages, dependent, stream);
+        case 32: return launch_stream_group<32>(grp, t_tiles, plan.split_k, plan.stages, dependent, stream);
+        case 64: return launch_stream_group<64>(grp, t_tiles, plan.split_k, plan.stages, dependent, stream);
+        case 128: return launch_stream_group<128>(grp, t_tiles, plan.split_k, plan.stages, dependent, stream);
+        case 256: return launch_stream_group<256>(grp, t_tiles, plan.split_k, plan.stages, dependent, stream);
         default: return ESP_ERR_INVALID_ARG;
     }
 }

@@ -402,3 +402,38 @@ def test_requested_ring_depth_of_the_streaming_kernel(M, K):
     from paper_2310_15929_b200 import binding as b
     with pytest.raises(b.EsparseError):
         spgemm(X, packed, theta, N, channel_major=True, kernel=4, pipeline_stages=1)
+
+
+@pytest.mark.parametrize("M", [16, 130, 520])
+@pytest.mark.parametrize("channel_major", [True, False])
+def test_grouped_products_in_one_call(M, channel_major):
+    """Three linears with their own weights, permutations, inputs and feature counts through esp_spgemm_grouped: one launch
+    of the streaming kernel up to 256 tokens, separate calls beyond; every output against the oracle's product."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    dev = torch.device("cuda:0")
+    K = 1160
+    Ns = [384, 200, 512]
+    g = np.random.default_rng(M)
+    probs = []
+    for N in Ns:
+        vals, meta, theta = pruned(N + M, N, K)
+        X = g.standard_normal((M, K)).astype(np.float16)
+        Xd = torch.from_numpy(X).to(dev)
+        if channel_major:
+            pad = torch.zeros(K, (M + 7) // 8 * 8, dtype=torch.float16, device=dev)
+            pad[:, :M] = Xd.t()
+            Xd = pad[:, :M]
+        probs.append(dict(vals=vals, meta=meta, theta=theta, X=X, Xd=Xd, packed=pack_on_gpu(vals, meta),
+                          th=torch.from_numpy(theta).to(dev), Y=torch.full((M, N), float("nan"), dtype=torch.float16, device=dev)))
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR if channel_major else b.ESP_X_TOKEN_MAJOR
+    nws = 3 * max(b.esp_spgemm_workspace_bytes(M, N, K, o) for N in Ns)
+    ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+    b.esp_spgemm_grouped([q["Xd"] for q in probs], [q["packed"] for q in probs], [q["th"] for q in probs],
+                         [q["Y"] for q in probs], o, ws)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    for q in probs:
+        check(q["Y"].cpu().numpy(), orc.product(q["X"], q["vals"], q["meta"], q["theta"]))
