@@ -2,7 +2,7 @@
 """Benchmark of the E-Sparse hot path on B200.
 
 A step is one forward pass over the seven pruned linears of a LLaMA-7B-shaped decoder layer
-(benchmark configs[1]) at M = 2048 tokens: seven esp_spgemm calls.  `value` is the dense-equivalent
+(workload 1 of paper_2310_15929_b200/inputs.py) at M = 2048 tokens: seven esp_spgemm calls.  `value` is the dense-equivalent
 throughput 2*M*N*K / t summed over the layer (the unit the sparse tensor-core peak is quoted in; executed
 flops are half of that).  The operands are produced on the device by esp_metric_prune from seeded synthetic
 weights and calibration activations before the timed region; that producer pass, the decode regime (M = 16,

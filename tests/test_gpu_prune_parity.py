@@ -98,7 +98,7 @@ def test_ablation_toggles(toggles):
 
 
 def test_config0_end_to_end():
-    """BASELINE config 0: 512x512 layer, 128 calibration tokens, 8 outlier channels x20."""
+    """Workload 0: 512x512 layer, 128 calibration tokens, 8 outlier channels x20."""
     from tests.gpu_util import GpuPrune
     wl = inputs.WORKLOADS[0]
     W, X = inputs.make_weight(wl, "fc"), inputs.make_calibration(wl, "fc")
