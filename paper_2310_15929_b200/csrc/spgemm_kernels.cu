@@ -1325,7 +1325,7 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
     }
     if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED) {
         if (bn == 0) {
-            // cost ~ waves of clusters x time of one channel step: the longer of the step's MMAs (8 x TN/2 clocks) and its
+            // cost ~ waves of clusters x time of one wave, in clocks: a channel step costs its MMAs (8 x TN/2 clocks) and its
             // 36 KB of weights + X tile (64-token blocks: 16 KB for TN = 128, else 32 KB) at the ~70 B/clk an SM pulls from
             // L2.  Wide tiles win once the grid fills the machine; a grid of less than one wave runs faster on narrow ones.
             const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
@@ -1333,7 +1333,9 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
             for (int tn : {240, 224, 192, 128}) {
                 const long clusters = f_pairs * ceil_div(M, tn);
                 const double mma = 4.0 * tn, copy = (36864.0 + (tn > 128 ? 32768.0 : 16384.0)) / 70.0;
-                const double cost = (double)ceil_div(clusters, per_wave) * (mma > copy ? mma : copy) * (k_tiles + 12.0);
+                // per wave: the channel steps (both terms show in the measured step time), an epilogue that grows with the
+                // tile (about ten steps' worth at 240 tokens) and a fixed set-up
+                const double cost = (double)ceil_div(clusters, per_wave) * (0.5 * (mma + copy) * k_tiles + 40.0 * tn + 2000.0);
                 if (best < 0.0 || cost < best) { best = cost; bn = tn; }
             }
         }
