@@ -1212,6 +1212,10 @@ __global__ void __launch_bounds__(256) transpose_x_kernel(const uint16_t *__rest
     __shared__ uint16_t tile[32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int k0 = blockIdx.x * 32, m0 = blockIdx.y * 32;
+    // As a programmatic dependent (static_weights): the GEMM behind this copy may start at once and prefetch its weights;
+    // X, and the workspace the preceding GEMM may still read, are touched only after that kernel is done.
+    grid_launch_dependents();
+    grid_dependency_wait();
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int m = m0 + ty + 8 * i, k = k0 + tx;
@@ -1223,6 +1227,20 @@ __global__ void __launch_bounds__(256) transpose_x_kernel(const uint16_t *__rest
         const int k = k0 + ty + 8 * i, m = m0 + tx;
         if (k < K && m < ldt) Xt[(long)k * ldt + m] = tile[tx][ty + 8 * i];
     }
+}
+
+static cudaError_t launch_transpose(const uint16_t *X, int M, int K, long ldx, uint16_t *Xt, long ldt, bool dependent,
+                                    cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ceil_div(K, 32), ceil_div(ldt, 32), 1);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, transpose_x_kernel, X, M, K, ldx, Xt, ldt);
 }
 
 // A wait nobody ends: one thread polls a barrier that receives no arrival, gives up after a short limit, records
@@ -1446,9 +1464,8 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             // token-major input: transposed (not permuted) copy into the caller's workspace
             const long ldt = transposed_ld(M);
             if (!workspace || workspace_bytes < (size_t)K * ldt * 2) return ESP_ERR_WORKSPACE;
-            transpose_x_kernel<<<dim3(ceil_div(K, 32), ceil_div(ldt, 32)), 256, 0, stream>>>(
-                reinterpret_cast<const uint16_t *>(X), M, K, ldx, reinterpret_cast<uint16_t *>(workspace), ldt);
-            ESP_CUDA_OK(cudaGetLastError());
+            ESP_CUDA_OK(launch_transpose(reinterpret_cast<const uint16_t *>(X), M, K, ldx, reinterpret_cast<uint16_t *>(workspace),
+                                         ldt, o.static_weights != 0, stream));
             p.X = reinterpret_cast<const __half *>(workspace);
             p.ldx = ldt;
             p.x_channel_major = 1;
@@ -1558,9 +1575,7 @@ esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, 
             if (o.x_layout != ESP_X_CHANNEL_MAJOR) {      // token-major: a transposed copy per problem, one after the other
                 const long ldt = transposed_ld(M);
                 uint16_t *xt = reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(workspace) + (size_t)i * tbytes);
-                transpose_x_kernel<<<dim3(ceil_div(K, 32), ceil_div(ldt, 32)), 256, 0, stream>>>(
-                    reinterpret_cast<const uint16_t *>(X[i]), M, K, ldx, xt, ldt);
-                ESP_CUDA_OK(cudaGetLastError());
+                ESP_CUDA_OK(launch_transpose(reinterpret_cast<const uint16_t *>(X[i]), M, K, ldx, xt, ldt, o.static_weights != 0, stream));
                 p.X = reinterpret_cast<const __half *>(xt);
                 p.ldx = ldt;
             }
