@@ -1572,10 +1572,14 @@ esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, 
         p.xflags = nullptr;
         grp.ft_start[i] = ft;
         if (i < count) {
-            if (o.x_layout != ESP_X_CHANNEL_MAJOR) {      // token-major: a transposed copy per problem, one after the other
+            if (o.x_layout != ESP_X_CHANNEL_MAJOR) {      // token-major: a transposed copy per distinct input, one after the other
                 const long ldt = transposed_ld(M);
-                uint16_t *xt = reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(workspace) + (size_t)i * tbytes);
-                ESP_CUDA_OK(launch_transpose(reinterpret_cast<const uint16_t *>(X[i]), M, K, ldx, xt, ldt, o.static_weights != 0, stream));
+                int first = i;
+                for (int e = 0; e < i; ++e)
+                    if (X[e] == X[i]) { first = e; break; }                 // same-input linears (q, k, v) share the copy
+                uint16_t *xt = reinterpret_cast<uint16_t *>(reinterpret_cast<uint8_t *>(workspace) + (size_t)first * tbytes);
+                if (first == i)
+                    ESP_CUDA_OK(launch_transpose(reinterpret_cast<const uint16_t *>(X[i]), M, K, ldx, xt, ldt, o.static_weights != 0, stream));
                 p.X = reinterpret_cast<const __half *>(xt);
                 p.ldx = ldt;
             }

@@ -437,3 +437,26 @@ def test_grouped_products_in_one_call(M, channel_major):
     assert b.esp_last_device_status() == b.ESP_OK
     for q in probs:
         check(q["Y"].cpu().numpy(), orc.product(q["X"], q["vals"], q["meta"], q["theta"]))
+
+
+def test_grouped_products_sharing_one_input():
+    """q, k, v style: three weights on the SAME token-major X (one transposed copy serves all three)."""
+    import torch
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu
+    dev = torch.device("cuda:0")
+    M, K, Ns = 16, 1160, [384, 200, 512]
+    X = np.random.default_rng(3).standard_normal((M, K)).astype(np.float16)
+    Xd = torch.from_numpy(X).to(dev)
+    probs = []
+    for N in Ns:
+        vals, meta, theta = pruned(N + 9, N, K)
+        probs.append(dict(vals=vals, meta=meta, theta=theta, packed=pack_on_gpu(vals, meta), th=torch.from_numpy(theta).to(dev),
+                          Y=torch.full((M, N), float("nan"), dtype=torch.float16, device=dev)))
+    o = b.esp_gemm_opts_default()
+    ws = torch.empty(3 * max(b.esp_spgemm_workspace_bytes(M, N, K, o) for N in Ns), dtype=torch.uint8, device=dev)
+    b.esp_spgemm_grouped([Xd] * 3, [q["packed"] for q in probs], [q["th"] for q in probs], [q["Y"] for q in probs], o, ws)
+    torch.cuda.synchronize()
+    assert b.esp_last_device_status() == b.ESP_OK
+    for q in probs:
+        check(q["Y"].cpu().numpy(), orc.product(X, q["vals"], q["meta"], q["theta"]))
