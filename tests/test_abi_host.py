@@ -156,3 +156,23 @@ def test_plan_table_round_trip(tmp_path):
     assert not b.apply_plan(o, loaded, 17, 4096, 4096)
     o2 = b.esp_gemm_opts_default()                       # another layout is another entry
     assert not b.apply_plan(o2, loaded, 16, 4096, 4096)
+
+
+def test_grouped_and_tune_argument_checks_need_no_device():
+    import ctypes
+    o = b.esp_gemm_opts_default()
+    one = (ctypes.c_void_p * 1)(0x1000)
+    n = (ctypes.c_int * 1)(128)
+    ld = (ctypes.c_long * 1)(128)
+    call = lambda count: b._lib.esp_spgemm_grouped(count, one, 16, 128, 128, one, one, n, one, ld, ctypes.byref(o), None, 0, None)
+    assert call(0) == b.ESP_ERR_INVALID_ARG
+    assert call(5) == b.ESP_ERR_INVALID_ARG
+    o.bias = 0x2000                                           # a common bias makes no sense for several weights
+    assert call(1) == b.ESP_ERR_INVALID_ARG
+    o.bias = None
+    o.pipeline_stages = 1
+    assert call(1) == b.ESP_ERR_INVALID_ARG
+    o.pipeline_stages = 0
+    best = ctypes.c_float()
+    assert b._lib.esp_spgemm_tune(None, 16, 128, 128, None, None, 128, None, 128, ctypes.byref(o), None, 0, 0,
+                                  ctypes.byref(best), None, None) == b.ESP_ERR_INVALID_ARG
