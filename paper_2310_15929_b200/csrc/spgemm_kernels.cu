@@ -1291,7 +1291,7 @@ static size_t ximg_bytes(int M, int K, int tn) {
 size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o) { return transpose_bytes(M, K, o); }
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
     size_t n = transpose_bytes(M, K, o);
-    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 256 && o.split_k <= 1);
+    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 1);
     if (pair_possible) {
         size_t img = 0;
         for (int tn : {128, 192, 224, 240}) img = std::max(img, ximg_bytes(M, K, tn));
@@ -1339,7 +1339,14 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
         else if (o.force_kernel == ESP_KERNEL_PAIR) g.kernel = ESP_KERNEL_PAIR;
         else if (o.force_kernel == ESP_KERNEL_PAIR_TILED) g.kernel = ESP_KERNEL_PAIR_TILED;
         else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
-        else g.kernel = (M > 256 && o.split_k <= 1) ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;   // the pair kernel has no K-slices
+        else {
+            // The pair kernel (no K-slices) takes every M > 256, and 64 < M <= 256 when the weight has enough feature tiles
+            // to give it twenty clusters or more: there it beats the streaming kernel's gather and K-slice reduction
+            // (11008 x 4096 at 128 / 256 tokens: 33 against 47 / 51 us), below that it leaves most SMs idle.
+            const long clusters128 = (long)ceil_div(f_tiles, 4) * ceil_div(M, 128);
+            const bool pair = o.split_k <= 1 && (M > 256 || (M > 64 && clusters128 >= 20));
+            g.kernel = pair ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;
+        }
     }
     if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED) {
         if (bn == 0) {
