@@ -175,13 +175,15 @@ enum { ESP_KERNEL_AUTO = 0,
                                     unit's row gather (correct, but that unit retires such gathers too
                                     slowly to feed the MMA; kept for comparison)                        */
        ESP_KERNEL_STREAM = 4,    /* channel-major X rows streamed by asynchronous 16-byte copies, weight
-                                    tiles by bulk copies; every token count (default up to 256 tokens)  */
+                                    tiles by bulk copies; every token count (default up to 256 tokens,
+                                    except where the pair kernel below is faster)                       */
        ESP_KERNEL_PAIR = 5,      /* large M: two SMs share one 512-feature x token_tile MMA tile
                                     (token_tile 240 by default; 128, 192, 224 or 256 on request); X rows
                                     are gathered through the permutation by 16-byte copies              */
        ESP_KERNEL_PAIR_TILED = 6 };/* the same tile, fed by bulk copies: a pass over X first writes the
                                     permuted, swizzled operand images into the workspace (default for
-                                    large M when the workspace has room; token_tile 128..240)           */
+                                    more than 256 tokens, and from 65 tokens on weights with many
+                                    feature tiles, when the workspace has room; token_tile 128..240)    */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */

@@ -310,8 +310,9 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
     struct Cand { int kernel, tile, split, stages; };
     std::vector<Cand> cands;
     cands.push_back({opts->force_kernel, opts->token_tile, opts->split_k, opts->pipeline_stages});
-    if (M > 256) {
+    if (M > 64) {
         for (int tile : {240, 224, 192, 128}) {
+            if (tile > 128 && M <= 128) continue;
             cands.push_back({ESP_KERNEL_PAIR_TILED, tile, 1, 0});
             cands.push_back({ESP_KERNEL_PAIR, tile, 1, 0});
         }
