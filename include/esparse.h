@@ -38,7 +38,7 @@ typedef enum {
     ESP_ERR_SHAPE = 2,         /* non-positive sizes, C % 8 != 0, leading dimension too small         */
     ESP_ERR_ALIGNMENT = 3,     /* a base pointer or leading dimension is not 16-byte aligned          */
     ESP_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than the *_workspace_bytes() answer       */
-    ESP_ERR_UNSUPPORTED = 5,   /* pattern other than 2:4, bins > 1024, device is not sm_100           */
+    ESP_ERR_UNSUPPORTED = 5,   /* pattern other than 2:4 / 4:8, bins > 512, device is not sm_100      */
     ESP_ERR_CUDA = 6,          /* a CUDA runtime call or a launch failed                              */
     ESP_ERR_TIMEOUT = 7,       /* a bounded in-kernel wait gave up (reported by esp_last_device_status) */
     ESP_ERR_STATIC_LIMIT = 8   /* esp_spgemm_static: the sizes need more than ESP_STATIC_SCRATCH_BYTES   */
@@ -57,7 +57,7 @@ int esp_version(void);
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_prune_opts)                                         */
     double alpha;                /* weight of the norm in Eq. 3; the paper gives no value             */
-    int bins;                    /* K of Eq. 1 (paper: 100); 2..1024                                  */
+    int bins;                    /* K of Eq. 1 (paper: 100); 2..512                                   */
     int n_keep, m_group;         /* N:M pattern: 2:4, or 4:8 (Table 1's second pattern: metric, global shuffle,
                                     selection and compression only -- use_lbs must be 0 and packed NULL,
                                     no tensor-core form exists; meta then holds one byte per group of 8,
@@ -81,7 +81,12 @@ typedef struct {
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_prune_stats)                                         */
     long long near_tie_groups;   /* groups whose 2nd and 3rd metric differ by < 1e-6 relative         */
+    long long near_tie_sort;     /* global shuffle: neighbours in rank whose mean metrics differ by < 1e-6
+                                    relative (0 when the shuffle is off or the order is given)        */
+    long long near_tie_swaps;    /* block shuffle: applied swaps whose gain beats the runner-up's by < 1e-6
+                                    relative                                                           */
     long long lbs_swaps_total;   /* swaps applied by the local block shuffle                          */
+    double obj_identity;         /* Eq. 5 objective (2 of every 4 kept) under the original channel order */
     double obj_after_gns;        /* Eq. 5 objective under the order after the global shuffle          */
     double obj_after_lbs;        /* Eq. 5 objective under the final order                             */
 } esp_prune_stats;

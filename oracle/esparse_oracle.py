@@ -171,7 +171,10 @@ def channel_mean_metric(W: np.ndarray, s: np.ndarray) -> np.ndarray:
     """Mean of xi over the No rows of each channel: (s_c * sum_j |W[j,c]|) / No.
     The column sum of |W| is taken exactly (integers of 2^-24), so it does not depend on row order."""
     No = W.shape[0]
-    colsum = abs_fixed(W).sum(axis=0)
+    colsum = np.zeros(W.shape[1], dtype=np.int64)
+    step = max(1, (1 << 24) // max(W.shape[1], 1))     # row blocks only bound the temporaries: integer sums are exact
+    for r0 in range(0, No, step):
+        colsum += abs_fixed(W[r0:r0 + step]).sum(axis=0)
     a = colsum.astype(np.float64) * _FIXED_SCALE
     return (np.asarray(s, dtype=np.float64) * a) / float(No)
 
@@ -392,8 +395,9 @@ def metric_prune(W: np.ndarray, xcal: np.ndarray, alpha: float, *, bins: int = B
     """norm -> entropy -> score -> global shuffle -> block shuffle -> 2:4 selection -> compression."""
     W = np.asarray(W, dtype=np.float16)
     C = W.shape[1]
-    am = channel_norm(xcal)
-    ir = channel_entropy(xcal, bins, global_bin_range)
+    # (with a supplied score the calibration activations are optional: the statistics are then not formed)
+    am = channel_norm(xcal) if xcal is not None else None
+    ir = channel_entropy(xcal, bins, global_bin_range) if xcal is not None else None
     s = channel_score(ir, am, alpha, use_entropy, use_norm) if score is None else np.asarray(score, np.float64)
     mean = channel_mean_metric(W, s)
     ident = np.arange(C, dtype=np.int32)

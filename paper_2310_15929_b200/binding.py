@@ -30,7 +30,8 @@ class esp_prune_opts(ctypes.Structure):
 
 
 class esp_prune_stats(ctypes.Structure):
-    _fields_ = [("struct_size", c_size_t), ("near_tie_groups", c_longlong), ("lbs_swaps_total", c_longlong),
+    _fields_ = [("struct_size", c_size_t), ("near_tie_groups", c_longlong), ("near_tie_sort", c_longlong),
+                ("near_tie_swaps", c_longlong), ("lbs_swaps_total", c_longlong), ("obj_identity", c_double),
                 ("obj_after_gns", c_double), ("obj_after_lbs", c_double)]
 
 
@@ -293,7 +294,7 @@ def esp_spgemm_static(X, packed, perm, Y, stream=None):
     out = ESP_OUT_F32 if Y.dtype == torch.float32 else ESP_OUT_F16
     st = esp_spgemm_static_raw(X, M, K, X.stride(0), packed, perm, N, Y, Y.stride(0), out, _stream(stream))
     if st != ESP_OK:
-        raise EsparseError(st, "esp_spgemm_static", "esp_spgemm_plan")
+        raise EsparseError(st, "esp_spgemm_static")
 
 
 def esp_selftest_wait_timeout(stream=None) -> None:

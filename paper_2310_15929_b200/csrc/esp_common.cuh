@@ -45,8 +45,9 @@ struct PruneWorkspace {
     unsigned int *counts;                                    // [C][bins]
     unsigned long long *colsum;                              // [C]
     int32_t *theta0;                                         // [C]
-    unsigned long long *counters;                            // [8]: 0 near-tie groups, 1 lbs swaps
-    double *objective;                                       // [2]: after gns, after lbs
+    unsigned long long *counters;                            // [8]: 0 near-tie groups, 1 lbs swaps, 2 near-ties of the sort, 3 of the swaps
+    double *objective;                                       // [4]: after gns, after lbs, identity order
+    double *sorted_mean;                                     // [C] channel means in rank order
     uint16_t *wt;                                            // [C][ldt] |W| bits, channel-major
     double *table;                                           // [nblocks][64][4][256]
     double *base;                                            // [C/4]

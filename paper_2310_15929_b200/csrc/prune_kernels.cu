@@ -258,7 +258,7 @@ __global__ void mean_metric_kernel(int C, int No, const unsigned long long *__re
 // a group).
 // --------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__restrict__ mean, int use_gns, int m_group,
-                                                       int32_t *__restrict__ theta0) {
+                                                       int32_t *__restrict__ theta0, double *__restrict__ sorted_mean) {
     __shared__ double tile[256];
     const int c = blockIdx.x * 256 + threadIdx.x;
     if (!use_gns) {
@@ -280,7 +280,23 @@ __global__ void __launch_bounds__(256) gns_rank_kernel(int C, const double *__re
     if (c < C) {
         const int G = C / m_group;
         theta0[(rank % G) * m_group + rank / G] = c;
+        sorted_mean[rank] = mine;
     }
+}
+
+// Near-ties of the sort: neighbours in rank whose means differ by less than 1e-6 relative (the order of such a pair
+// hangs on the last bits of the score).  counters[2] receives the count.
+__global__ void __launch_bounds__(256) gns_near_tie_kernel(int C, const double *__restrict__ sorted_mean,
+                                                           unsigned long long *__restrict__ counters) {
+    const int r = blockIdx.x * 256 + threadIdx.x;
+    unsigned int near = 0;
+    if (r + 1 < C) {
+        const double a = sorted_mean[r], b = sorted_mean[r + 1];
+        near = __dsub_rn(a, b) < __dmul_rn(1e-6, fabs(a)) ? 1u : 0u;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) near += __shfl_xor_sync(0xFFFFFFFFu, near, off);
+    if ((threadIdx.x & 31) == 0 && near) atomicAdd(&counters[2], (unsigned long long)near);
 }
 
 // --------------------------------------------------------------------------------------------------
@@ -530,7 +546,7 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
     __shared__ int pos2x[kLbsMax];
     __shared__ int chan[kLbsMax];
     __shared__ double s_base[kLbsGroups];
-    __shared__ double red_gain[16];
+    __shared__ double red_gain[16], red_second[16];
     __shared__ int red_idx[16];
     __shared__ int decision;      // linear pair index i*256+j, or -1 to stop
     __shared__ unsigned long long s_B[4];
@@ -539,8 +555,9 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
     if (tid < G) s_base[tid] = base[p0 / 4 + tid];
     __syncthreads();
     int swaps = 0;
+    int near_swaps = 0;                                        // kept by thread 0 only
     for (;;) {
-        double best = -INFINITY;
+        double best = -INFINITY, second = -INFINITY;           // second: largest gain once one instance of the best is set aside
         int best_e = 0x7FFFFFFF;
         if (max_swaps <= 0 || swaps < max_swaps) {
             for (int e = tid; e < kLbsMax * kLbsMax; e += 512) {
@@ -550,27 +567,39 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
                 // rows of the table are rewritten by other CTAs of the cluster: read them from L2, never from this SM's L1
                 double after = __dadd_rn(__ldcg(&tb[(gi * 4 + si) * kLbsMax + pos2x[j]]), __ldcg(&tb[(gj * 4 + sj) * kLbsMax + pos2x[i]]));
                 double gain = __dsub_rn(after, __dadd_rn(s_base[gi], s_base[gj]));
-                if (gain > best || (gain == best && e < best_e)) { best = gain; best_e = e; }
+                if (gain > best || (gain == best && e < best_e)) { second = fmax(second, best); best = gain; best_e = e; }
+                else second = fmax(second, gain);
             }
         }
+        // merging two (best, second) pairs: the larger best wins (ties: smaller pair index), the loser's best competes
+        // with both seconds -- the result is the second-largest of the union whatever the order of merging
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             double og = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+            double os = __shfl_xor_sync(0xFFFFFFFFu, second, off);
             int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
+            second = fmax(fmax(second, os), fmin(best, og));
             if (og > best || (og == best && oe < best_e)) { best = og; best_e = oe; }
         }
-        if (lane == 0) { red_gain[warp] = best; red_idx[warp] = best_e; }
+        if (lane == 0) { red_gain[warp] = best; red_second[warp] = second; red_idx[warp] = best_e; }
         __syncthreads();
         if (warp == 0) {
             best = lane < 16 ? red_gain[lane] : -INFINITY;
+            second = lane < 16 ? red_second[lane] : -INFINITY;
             best_e = lane < 16 ? red_idx[lane] : 0x7FFFFFFF;
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 double og = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+                double os = __shfl_xor_sync(0xFFFFFFFFu, second, off);
                 int oe = __shfl_xor_sync(0xFFFFFFFFu, best_e, off);
+                second = fmax(fmax(second, os), fmin(best, og));
                 if (og > best || (og == best && oe < best_e)) { best = og; best_e = oe; }
             }
-            if (lane == 0) decision = (best > 0.0) ? best_e : -1;
+            if (lane == 0) {
+                decision = (best > 0.0) ? best_e : -1;
+                // an applied swap whose runner-up is within 1e-6 relative: counted, not acted on
+                if (best > 0.0 && second > -INFINITY && __dsub_rn(best, second) < __dmul_rn(1e-6, fabs(best))) ++near_swaps;
+            }
         }
         __syncthreads();
         const int d = decision;
@@ -616,6 +645,7 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
     if (tid < m) theta[p0 + tid] = chan[pos2x[tid]];
     if (tid < G) base[p0 / 4 + tid] = s_base[tid];
     if (tid == 0 && swaps) atomicAdd(&counters[1], (unsigned long long)swaps);
+    if (tid == 0 && near_swaps) atomicAdd(&counters[3], (unsigned long long)near_swaps);
 }
 
 // Sum of the group values in group order (Eq. 5 objective), one thread: deterministic.
@@ -627,14 +657,17 @@ __global__ void objective_kernel(int G, const double *__restrict__ base, double 
     }
 }
 
-// base[g] = V(g) under theta for every group (used when the block shuffle is off but stats are wanted).
+// base[g] = V(g) under theta for every group (the objective of an order that the block shuffle does not produce itself).
 __global__ void __launch_bounds__(256) group_values_kernel(const uint16_t *__restrict__ Wt, long ldt,
                                                            const double *__restrict__ score,
                                                            const int32_t *__restrict__ theta, int G,
                                                            double *__restrict__ base) {
     const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (g >= G) return;
-    double v = group_value_warp(Wt, ldt, score, theta[4 * g], theta[4 * g + 1], theta[4 * g + 2], theta[4 * g + 3]);
+    int c[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) c[k] = theta ? theta[4 * g + k] : 4 * g + k;      // NULL: the identity order
+    double v = group_value_warp(Wt, ldt, score, c[0], c[1], c[2], c[3]);
     if ((threadIdx.x & 31) == 0) base[g] = v;
 }
 
@@ -863,7 +896,8 @@ PruneWorkspace carve_prune_workspace(void *ws, int No, int C, int T, const esp_p
     w.colsum = (unsigned long long *)take(sizeof(unsigned long long) * C);
     w.theta0 = (int32_t *)take(sizeof(int32_t) * C);
     w.counters = (unsigned long long *)take(sizeof(unsigned long long) * 8);
-    w.objective = (double *)take(sizeof(double) * 2);
+    w.objective = (double *)take(sizeof(double) * 4);
+    w.sorted_mean = (double *)take(sizeof(double) * C);
     w.ldt = (long)align_up((size_t)No, 256);
     w.wt = (uint16_t *)take(sizeof(uint16_t) * (size_t)C * w.ldt);
     int nblocks = ceil_div(C, o.lbs_block > 0 ? o.lbs_block : kLbsMax);
@@ -956,7 +990,7 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     const int cthreads = 256;
     const int cblocks = ceil_div(C, cthreads);
     ESP_CUDA_OK(cudaMemsetAsync(w.counters, 0, sizeof(unsigned long long) * 8, stream));
-    ESP_CUDA_OK(cudaMemsetAsync(w.objective, 0, sizeof(double) * 2, stream));
+    ESP_CUDA_OK(cudaMemsetAsync(w.objective, 0, sizeof(double) * 4, stream));
 
     const bool need_stats_pass = (o.score_override == nullptr) || chan_norm || chan_entropy;
     if (need_stats_pass && Xcal) {
@@ -996,14 +1030,20 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     int32_t *theta0 = (o.use_lbs || stats) ? w.theta0 : perm;
     if (o.perm_override)
         ESP_CUDA_OK(cudaMemcpyAsync(theta0, o.perm_override, sizeof(int32_t) * C, cudaMemcpyDeviceToDevice, stream));
-    else
-        gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, o.m_group, theta0);
+    else {
+        gns_rank_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.mean, o.use_gns, o.m_group, theta0, w.sorted_mean);
+        if (o.use_gns && stats) gns_near_tie_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, w.sorted_mean, w.counters);
+    }
     ESP_CUDA_OK(cudaGetLastError());
 
     // K5
     const int G = C / 4;
     if (o.use_lbs || stats) {
         abs_transpose_kernel<<<dim3(ceil_div(C, 32), ceil_div(w.ldt, 32)), 256, 0, stream>>>(W, No, C, ldw, w.wt, w.ldt);
+    }
+    if (stats) {                             // Eq. 5 under the identity order (w.base is rewritten below)
+        group_values_kernel<<<ceil_div(G, 8), 256, 0, stream>>>(w.wt, w.ldt, w.score, nullptr, G, w.base);
+        objective_kernel<<<1, 32, 0, stream>>>(G, w.base, w.objective + 2);
     }
     if (o.use_lbs) {
         const int nblocks = ceil_div(C, o.lbs_block);
@@ -1055,12 +1095,15 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     }
     if (stats) {
         unsigned long long h_counters[8];
-        double h_obj[2];
+        double h_obj[4];
         ESP_CUDA_OK(cudaMemcpyAsync(h_counters, w.counters, sizeof(h_counters), cudaMemcpyDeviceToHost, stream));
         ESP_CUDA_OK(cudaMemcpyAsync(h_obj, w.objective, sizeof(h_obj), cudaMemcpyDeviceToHost, stream));
         ESP_CUDA_OK(cudaStreamSynchronize(stream));
         stats->near_tie_groups = (long long)h_counters[0];
+        stats->near_tie_sort = (long long)h_counters[2];
+        stats->near_tie_swaps = (long long)h_counters[3];
         stats->lbs_swaps_total = (long long)h_counters[1];
+        stats->obj_identity = h_obj[2];
         stats->obj_after_gns = h_obj[0];
         stats->obj_after_lbs = h_obj[1];
     }

@@ -86,6 +86,14 @@ def test_prune_argument_errors():
     assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED                         # 4:8 has no sparse MMA form
     o = b.esp_prune_opts_default(); o.bins = 5000
     assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED
+    # the documented range of bins is 2..512, at the boundary exactly
+    o = b.esp_prune_opts_default(); o.bins = 513
+    assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED
+    assert b.esp_metric_prune_workspace_bytes(512, 512, 128, o) == 0 and b.esp_calib_state_bytes(512, 513) == 0
+    o.bins = 512
+    assert b.esp_metric_prune_workspace_bytes(512, 512, 128, o) > 0 and b.esp_calib_state_bytes(512, 512) > 0
+    o.bins = 1
+    assert prune_call(opts=o) == b.ESP_ERR_UNSUPPORTED
     o = b.esp_prune_opts_default(); o.lbs_block = 250
     assert prune_call(opts=o) == b.ESP_ERR_INVALID_ARG
     o = b.esp_prune_opts_default(); o.struct_size = 8

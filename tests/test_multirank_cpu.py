@@ -44,3 +44,29 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(1.5, None, None) == 1.5
     assert bench.whole_job_rate(10.0, 1, 1000.0) == pytest.approx(10.0)
+
+
+def test_gpus_flag_must_agree_with_the_launcher():
+    """bench.py --gpus N under a launcher that started another number of ranks refuses to run (before touching a GPU)."""
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="4", RANK="0", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2"], env=env, capture_output=True, text=True)
+    assert r.returncode != 0
+    assert "4 ranks" in r.stderr
+
+
+def test_gpus_flag_without_a_launcher_starts_the_ranks_itself():
+    """--gpus 2 with no launcher around: bench.py starts two ranks; on the reference arm (CPU only) rank 0 prints the one
+    JSON line and the other rank exits 0 without work."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0", "--cpu-rows", "2", "--cpu-features", "16"], env=env, capture_output=True, text=True,
+                       timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["cpu_baseline"]["kind"] == "oracle"
+    assert out["e2e"]["h2d_bytes_per_step"] == 0

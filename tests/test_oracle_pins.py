@@ -206,6 +206,58 @@ def test_gns_bijection_quartiles_and_stability():
     assert np.all(np.abs(np.diff(np.sort(rank[theta0].reshape(64, 4), axis=1), axis=1)) == 64)
 
 
+def test_gns_near_tie_count_against_constructed_gaps():
+    """The near-tie counter of the sort: exactly the neighbours in rank closer than 1e-6 relative."""
+    base = np.array([8.0, 7.0, 6.0, 5.0, 4.0, 3.0, 2.0, 1.0])
+    _, near = orc.global_naive_shuffle(base)
+    assert near == 0                                          # well separated
+    m = base.copy()
+    m[5] = m[2] * (1.0 - 1e-7)                                # channel 5 lands right behind channel 2, 1e-7 apart
+    _, near = orc.global_naive_shuffle(m)
+    assert near == 1
+    m[7] = m[0] * (1.0 - 5e-7)                                # a second close pair at the top
+    _, near = orc.global_naive_shuffle(m)
+    assert near == 2
+    m = base.copy()
+    m[5] = m[2] * (1.0 - 1e-5)                                # ten times the threshold: not a near-tie
+    _, near = orc.global_naive_shuffle(m)
+    assert near == 0
+    m = base.copy()
+    m[6] = m[1]                                               # an exact tie counts (gap 0), order by channel index
+    theta0, near = orc.global_naive_shuffle(m)
+    assert near == 1
+    order = np.argsort(-m, kind="stable")
+    assert order.tolist().index(1) + 1 == order.tolist().index(6)
+    # brute force on a random input: count the close neighbours of the sorted list directly
+    g = np.random.default_rng(81)
+    mean = np.round(g.random(4096), 4) + 1.0                  # many exact and near ties
+    _, near = orc.global_naive_shuffle(mean)
+    srt = sorted(mean.tolist(), reverse=True)
+    assert near == sum(1 for a, b in zip(srt[:-1], srt[1:]) if a - b < 1e-6 * abs(a))
+    assert near > 0
+
+
+def test_gns_groups_of_eight_closed_form():
+    """m_group = 8 (the 4:8 pattern): rank r goes to group r mod G, slot r div G with G = C / 8."""
+    C = 64
+    G = C // 8
+    t, near = orc.global_naive_shuffle(-np.arange(C, dtype=np.float64), m_group=8)
+    p = np.arange(C)
+    assert np.array_equal(t, (p % 8) * G + p // 8)
+    assert near == 0
+    t16, _ = orc.global_naive_shuffle(np.arange(16, 0, -1).astype(np.float64), m_group=8)
+    assert t16.tolist() == [0, 2, 4, 6, 8, 10, 12, 14, 1, 3, 5, 7, 9, 11, 13, 15]
+    g = np.random.default_rng(82)
+    mean = g.random(256)
+    theta0, _ = orc.global_naive_shuffle(mean, m_group=8)
+    assert sorted(theta0.tolist()) == list(range(256))
+    rank = np.empty(256, dtype=np.int64)
+    rank[np.argsort(-mean, kind="stable")] = np.arange(256)
+    octile = rank[theta0].reshape(32, 8) // 32
+    assert np.all(octile == np.arange(8)[None, :])            # slot k of every group holds a channel of rank octile k
+    assert np.all(np.diff(rank[theta0].reshape(32, 8), axis=1) == 32)
+
+
 def test_channel_mean_matches_plain_mean_of_metric():
     W, X = rand_layer(9, 200, 48, 100)
     s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.3)
@@ -296,6 +348,54 @@ def test_lbs_vs_exhaustive_optimum_on_8_channels():
             hits += 1
         assert got >= one_swap * (1 - 1e-13) or got >= naive_objective(W, s, theta0)
     assert hits >= 1
+
+
+def _pair_gains_naive(W, s, theta, lo, hi):
+    base = naive_objective(W, s, theta)
+    gains = []
+    for i, j in itertools.combinations(range(lo, hi), 2):
+        if i // 4 == j // 4:
+            continue
+        t2 = theta.copy()
+        t2[i], t2[j] = t2[j], t2[i]
+        gains.append(naive_objective(W, s, t2) - base)
+    return sorted(gains, reverse=True)
+
+
+def test_lbs_near_tie_swaps_counted_against_brute_force():
+    """The counter of near-tied swaps: an applied swap whose gain beats the runner-up by less than 1e-6 relative.
+    (a) mirrored halves make every gain appear twice, so every applied swap is an exact tie with its mirror image;
+    (b) on a generic input the count equals the one found by replaying the swaps and ranking all pair gains naively."""
+    g = np.random.default_rng(83)
+    half = (g.standard_normal((20, 8)) * 0.02).astype(np.float16)
+    W = np.concatenate([half, half], axis=1)                  # channels 8..15 are copies of channels 0..7
+    s8 = 1.0 + g.random(8)
+    s = np.concatenate([s8, s8])
+    theta0 = np.arange(16, dtype=np.int32)
+    _, one = orc.local_block_shuffle(W, s, theta0, block=16, max_swaps=1)
+    if one.swaps_total == 1:
+        assert one.near_tie_swaps == 1
+    else:                                                     # no improving swap at all: nothing applied, nothing counted
+        assert one.near_tie_swaps == 0
+    assert one.swaps_total == 1, "the constructed input should have an improving swap"
+    # (b) generic input
+    for seed in (84, 85):
+        W, X = rand_layer(seed, 24, 16, 64)
+        s = orc.channel_score(orc.channel_entropy(X), orc.channel_norm(X), 0.2)
+        theta0 = np.arange(16, dtype=np.int32)
+        _, info = orc.local_block_shuffle(W, s, theta0, block=16)
+        expected, decided = 0, True
+        for k in range(info.swaps_total):
+            tk = theta0 if k == 0 else orc.local_block_shuffle(W, s, theta0, block=16, max_swaps=k)[0]   # (a cap of 0 means none)
+            gains = _pair_gains_naive(W, s, tk, 0, 16)
+            rel = (gains[0] - gains[1]) / abs(gains[0])
+            if 1e-8 < rel < 1e-4:
+                decided = False                               # too close to the threshold for the naive fp64 sums to tell
+            expected += 1 if rel < 1e-6 else 0
+        assert info.swaps_total > 0
+        if decided:
+            assert info.near_tie_swaps == expected
+    assert 0 <= info.near_tie_swaps <= info.swaps_total
 
 
 def _one_swap_orders(theta0):
