@@ -43,8 +43,7 @@ __global__ void __launch_bounds__(256) colstats_kernel(const __half *__restrict_
 #pragma unroll
     for (int k = 0; k < 8; ++k) { acc[k] = 0.0; mn[k] = INFINITY; mx[k] = -INFINITY; }
     if (c0 < C) {
-        for (int r = r_begin + ty; r < r_end; r += 8) {
-            uint4 v = __ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0));
+        auto add_row = [&](const uint4 &v) {
             const __half *h = reinterpret_cast<const __half *>(&v);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -53,7 +52,17 @@ __global__ void __launch_bounds__(256) colstats_kernel(const __half *__restrict_
                 mn[k] = fminf(mn[k], f);
                 mx[k] = fmaxf(mx[k], f);
             }
+        };
+        // rows in the same order as a plain loop (the order of the fp64 additions is part of the result), four loads in flight
+        int r = r_begin + ty;
+        for (; r + 24 < r_end; r += 32) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldg(reinterpret_cast<const uint4 *>(X + (long)(r + 8 * u) * ldx + c0));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) add_row(v[u]);
         }
+        for (; r < r_end; r += 8) add_row(__ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0)));
     }
     __shared__ double s_acc[8][256 + 1];
     __shared__ float s_mn[8][256 + 1], s_mx[8][256 + 1];
@@ -155,7 +164,13 @@ __global__ void __launch_bounds__(256) histogram_kernel(const __half *__restrict
     const int r_begin = blockIdx.y * rows_per_split;
     const int r_end = min(T, r_begin + rows_per_split);
     if (c0 < C) {
+        // Exact bin: floor of the fp64 quotient (x - lo) * K / (hi - lo).  Almost every element gets there in fp32: with lo
+        // exact in fp32 and r = K / (hi - lo) rounded once, q32 = (x - lo) * r is within 3 * 2^-24 relative of the exact
+        // quotient, i.e. within K * 1.8e-7 absolute, so wherever q32 sits further than eps = K * 2^-21 from an integer its
+        // floor IS the exact bin.  The elements that sit closer (about one in ten thousand, and always the channel's
+        // minimum and maximum) take the fp64 division.
         double l[8], scale_den[8];
+        float lf[8], rf[8];
         bool flat[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -163,19 +178,38 @@ __global__ void __launch_bounds__(256) histogram_kernel(const __half *__restrict
             double rng = __dsub_rn(hi[c0 + k], l[k]);
             flat[k] = !(rng > 0.0);
             scale_den[k] = flat[k] ? 1.0 : rng;
+            lf[k] = (float)l[k];                                   // exact when the range is a channel's own (an fp16 value)
+            const bool lo_exact = (double)lf[k] == l[k];
+            rf[k] = (flat[k] || !lo_exact) ? 0.f : (float)((double)bins / rng);   // 0: every element takes the fp64 path
         }
         const double kb = (double)bins;
-        for (int r = r_begin + ty; r < r_end; r += 32) {
-            uint4 v = __ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0));
+        const float eps = (float)bins * 0x1p-21f;
+        auto count_row = [&](const uint4 &v) {
             const __half *h = reinterpret_cast<const __half *>(&v);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-                double x = (double)__half2float(h[k]);
-                double q = __ddiv_rn(__dmul_rn(__dsub_rn(x, l[k]), kb), scale_den[k]);
-                int b = flat[k] ? 0 : min(bins - 1, (int)floor(q));
+                const float xf = __half2float(h[k]);
+                const float qf = (xf - lf[k]) * rf[k];
+                const float fl = floorf(qf);
+                const float fr = qf - fl;
+                int b = (int)fl;
+                if (!(fr > eps && fr < 1.f - eps)) {
+                    const double q = __ddiv_rn(__dmul_rn(__dsub_rn((double)xf, l[k]), kb), scale_den[k]);
+                    b = flat[k] ? 0 : max(0, min(bins - 1, (int)floor(q)));   // (the clamp at 0 only keeps a NaN in bounds)
+                }
                 atomicAdd(&s_cnt[(cl + k) * bins + b], 1u);
             }
+        };
+        // four rows per thread in flight
+        int r = r_begin + ty;
+        for (; r + 96 < r_end; r += 128) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldg(reinterpret_cast<const uint4 *>(X + (long)(r + 32 * u) * ldx + c0));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) count_row(v[u]);
         }
+        for (; r < r_end; r += 32) count_row(__ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0)));
     }
     __syncthreads();
     for (int i = threadIdx.x; i < 64 * bins; i += 256) {

@@ -309,8 +309,23 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                              // 0 = leader
-    const int pair_idx = (int)blockIdx.x >> 1;
-    const int tok0 = (int)blockIdx.y * TN;                                // first token of the pair's tile
+    // Cluster -> tile.  Clusters start in the order of their linear index (x fastest).  Taken row by row, one wave of
+    // clusters would span every feature pair on one or two token tiles, i.e. stream the whole weight from HBM once per
+    // wave.  With p.raster_panel = P > 1 the index runs down panels of P token tiles instead (P tiles of one feature pair,
+    // then the next pair): a wave then covers about 74 / P feature pairs x P token tiles, whose weight tiles and X images
+    // together stay in L2 while the wave runs.
+    int pair_idx = (int)blockIdx.x >> 1;
+    int ttile = (int)blockIdx.y;
+    if (p.raster_panel > 1) {
+        const int f_pairs = (int)gridDim.x >> 1, t_tiles = (int)gridDim.y;
+        const int c = ttile * f_pairs + pair_idx;
+        const int per_panel = p.raster_panel * f_pairs;
+        const int panel = c / per_panel, r = c - panel * per_panel;
+        const int height = min(p.raster_panel, t_tiles - panel * p.raster_panel);
+        pair_idx = r / height;
+        ttile = panel * p.raster_panel + (r - pair_idx * height);
+    }
+    const int tok0 = ttile * TN;                                          // first token of the pair's tile
     const int tok_cta = tok0 + (int)rank * L::kHalf;                      // first token this CTA stages
     const int nk = p.k_tiles;
     const int f_tiles = (p.N + 127) / 128;
@@ -436,12 +451,12 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             if (lane == 0 && iw < kCopies * STAGES) {
                 const int s = iw / kCopies, kind = iw % kCopies;
                 const bool is_x = kind == NA;
-                const uint32_t *xflag = p.xflags + (size_t)(blockIdx.y * 2 + rank) * nk;
+                const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * nk;
                 if (is_x || present[kind]) {
                     const uint32_t bytes = is_x ? (uint32_t)L::kXStage : (uint32_t)kTileBytes;
                     constexpr int kRowBytes = 1024;                       // the tensor maps see both buffers as 1024-byte rows
                     const CUtensorMap *map = is_x ? &xmap : &wmap;
-                    const int row0 = is_x ? (int)((blockIdx.y * 2 + rank) * nk) * (L::kXStage / kRowBytes)
+                    const int row0 = is_x ? (int)((ttile * 2 + rank) * nk) * (L::kXStage / kRowBytes)
                                           : ftile[kind] * nk * (kTileBytes / kRowBytes);
                     const int row_step = (int)bytes / kRowBytes;
                     const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
