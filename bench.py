@@ -709,12 +709,14 @@ def run_profile_case(args):
     case = args.profile_case
     N, K = (4096, 4096)
     if case == "prune":
+        # the producer on a slice of the LLaMA-7B-shaped q projection: all 4096 input channels and all 32768 calibration
+        # tokens (268 MB of activations: larger than L2), 1024 output rows, one block-shuffle swap per block
         from paper_2310_15929_b200 import inputs
         wl = inputs.WORKLOADS[WORKLOAD]
-        T = 4096
+        T = wl.calib_tokens
         W = torch.from_numpy(inputs.make_weight(wl, "q", No=1024)).to(dev)
         Xc = torch.from_numpy(inputs.make_calibration(wl, "q", T=T)).to(dev)
-        o = b.esp_prune_opts_default(); o.alpha = 1.0 / math.sqrt(T); o.lbs_max_swaps = 2
+        o = b.esp_prune_opts_default(); o.alpha = 1.0 / math.sqrt(T); o.lbs_max_swaps = 1
         ws = torch.empty(b.esp_metric_prune_workspace_bytes(1024, K, T, o), dtype=torch.uint8, device=dev)
         vals = torch.empty(1024, K // 2, dtype=torch.float16, device=dev)
         meta = torch.empty(1024, K // 8, dtype=torch.uint8, device=dev)
@@ -722,9 +724,9 @@ def run_profile_case(args):
         packed = torch.empty(b.esp_packed_bytes(1024, K), dtype=torch.uint8, device=dev)
         fn = lambda: b.esp_metric_prune(W, Xc, o, vals, meta, perm, packed, workspace=ws)
         ms = time_steps(fn, 2, 1)
-        print(json.dumps({"case": case, "No": 1024, "C": K, "T": T, "ms": ms}))
+        print(json.dumps({"case": case, "No": 1024, "C": K, "T": T, "ms": ms, "xcal_bytes": 2 * T * K}))
         return
-    M = PREFILL_M if case == "prefill" else DECODE_M
+    M = PREFILL_M if case == "prefill" else 128 if case == "mid" else DECODE_M
     vals = (torch.randn(N, K // 2, device=dev) * 0.02).half()
     meta = torch.full((N, K // 8), 0xE4, dtype=torch.uint8, device=dev)
     packed = torch.empty(b.esp_packed_bytes(N, K), dtype=torch.uint8, device=dev)
@@ -834,7 +836,7 @@ def main():
     ap.add_argument("--cpu-features", type=int, default=CPU_FEATURES)
     ap.add_argument("--eager", action="store_true", help="time plain esp_spgemm calls instead of a CUDA graph of the step")
     ap.add_argument("--quick", action="store_true", help="headline only: skip the decode, LLaMA-7B, per-config and producer sections")
-    ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "prune"],
+    ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "mid", "prune"],
                     help="run a few launches of one small case (for ncu) instead of the benchmark")
     ap.add_argument("--table5", action="store_true", help="time the GEMM shapes of the paper's Table 5 instead of the benchmark")
     args = ap.parse_args()

@@ -313,8 +313,10 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
     if (M > 64) {
         for (int tile : {240, 224, 192, 128}) {
             if (tile > 128 && M <= 128) continue;
-            cands.push_back({ESP_KERNEL_PAIR_TILED, tile, 1, 0});
-            cands.push_back({ESP_KERNEL_PAIR, tile, 1, 0});
+            for (int split = 1; split <= (tile == 128 ? 4 : 1); ++split) {      // K-slices: 128-token tiles only
+                cands.push_back({ESP_KERNEL_PAIR_TILED, tile, split, 0});
+                cands.push_back({ESP_KERNEL_PAIR, tile, split, 0});
+            }
         }
         cands.push_back({ESP_KERNEL_PAIR, 256, 1, 0});
     }
@@ -341,6 +343,7 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
         if (i > 0 && cands[i].kernel == ESP_KERNEL_STREAM &&
             (plan.split_k != cands[i].split || (cands[i].stages != 0 && plan.stages != cands[i].stages)))
             continue;                                                          // stepped down or clamped: a duplicate
+        if (i > 0 && cands[i].kernel != ESP_KERNEL_STREAM && plan.split_k != cands[i].split) continue;
         // one untimed call (first-use set-up, caches), then `reps` timed ones
         st = esp_spgemm(X, M, K, ldx, packed, perm, N, Y, ldy, &o, workspace, workspace_bytes, cuda_stream);
         if (st != ESP_OK) {

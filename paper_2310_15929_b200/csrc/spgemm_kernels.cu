@@ -612,12 +612,16 @@ __global__ void __launch_bounds__(192) spgemm_tma_kernel(const GemmParams p, con
 // touches only the weights and the permutation -- overlaps the predecessor's tail, and only the X rows
 // wait for it (griddepcontrol.wait).
 //
-// K is split across the CTAs of a cluster.  Partial tiles are reduced by pushing: token t of the tile is
-// owned by cluster rank t % split; every CTA stores its fp32 partial rows straight into the owner's
-// shared memory (slot = sender's rank) and arrives on the owner's mbarrier; the owner adds the slots in
-// rank order -- deterministic, no global scratch, one cluster-wide rendezvous at start-up only.  (Token tiles
-// of 64 and more, whose partial tiles would crowd out the stages, stage them in the stage area after the
-// main loop and let each owner pull its rows from the peers instead.)
+// K is split across the CTAs of a cluster.  Partial tiles are reduced by pushing: the tile's tokens are dealt to the
+// cluster ranks in contiguous runs of `cnt4` rows (a multiple of 4, so that four accumulator columns always go to one
+// owner as one 16-byte store); every CTA sends its fp32 partial rows straight into the owner's shared memory with
+// asynchronous remote stores (slot = sender's rank) that complete on the owner's mbarrier; the owner adds the slots in
+// rank order -- deterministic, no global scratch.  Token tiles up to 32 keep a receive area of their own and push as
+// soon as their accumulator is complete; wider tiles, whose partials would crowd out the ring, receive into the ring
+// itself once a cluster barrier has told every CTA that all MMAs of the cluster are done reading it.  (Measured on
+// 4096 x 4096 at 128 tokens: owners pulling the rows from their peers with remote loads took 8.4 us for 64 KB per CTA;
+// element-wise pushes for slice counts that are not a power of two took 10 us at 32 tokens.  The 16-byte pushes take
+// about 1.5 us.)
 // grid (feature tiles, token tiles, split_k), cluster (1,1,split_k), block 192:
 //   warp 0 lane 0  weight-tile producer        warp 1  tensor-memory allocation; lane 0: tcgen05.cp + sparse MMAs
 //   warps 2..5     X row producers, then epilogue (one quarter of the accumulator lanes each)
@@ -704,38 +708,22 @@ struct StreamCfg {
     static constexpr int kStage = kTileBytes + kXStage;              // a multiple of 1024
     static constexpr uint32_t kLayout = BN >= 64 ? 2u : BN == 32 ? 4u : 6u;   // 128 / 64 / 32-byte swizzle
     static constexpr int kSwzShift = BN >= 64 ? 0 : BN == 32 ? 1 : 2;         // row bits that feed the XOR
-    static constexpr bool kPush = BN <= 32;                          // K-slice reduction by pushing (else by pulling)
+    static constexpr bool kEarlyPush = BN <= 32;                     // partial rows pushed into a receive area of their own
     // 16-byte asynchronous row copies deliver 25 / 44 / 60 GB/s per SM from 128 / 256 / 512 threads: wide X tiles get
     // sixteen producer warps, narrow ones (little X per weight tile) four
     static constexpr int kProd = BN >= 64 ? 512 : 128;
     static constexpr int kThreads = 64 + kProd;
-    static constexpr int kRecvBytes = kPush ? (BN + 8) * 512 : 0;    // pushed partials: [sender][128 features][rows per owner] fp32
 };
-inline size_t stream_recv_bytes(int bn, int split) { return (split > 1 && bn <= 32) ? (size_t)(bn + 8) * 512 : 0; }
+// Rows of a token tile that one cluster rank owns in the K-slice reduction (a multiple of 4; rank o owns rows
+// [o * cnt4, (o + 1) * cnt4) of the tile, clipped to the tile).
+__host__ __device__ inline int stream_cnt4(int bn, int split) { return (((bn + split - 1) / split) + 3) & ~3; }
+// Pushed partials at one owner: [sender][group of 4 rows][128 features][4 rows] fp32.
+inline size_t stream_push_bytes(int bn, int split) { return split > 1 ? (size_t)split * stream_cnt4(bn, split) * 512 : 0; }
+inline size_t stream_recv_bytes(int bn, int split) { return bn <= 32 ? stream_push_bytes(bn, split) : 0; }   // beside the ring
 inline size_t stream_smem_bytes(int bn, int stages, int split) {
-    return (size_t)stages * (kTileBytes + 256 * bn) + stream_recv_bytes(bn, split) + kPermRing * 512 + 512 + 1024;
-}
-
-// Sends the 16 accumulator columns c0 .. c0+15 of this thread's feature to their owners (row % SPLIT), SPLIT a
-// power of two: the rows one owner gets from these 16 are consecutive in its slot, so they go as one vector.
-template <int SPLIT>
-__device__ __forceinline__ void push_columns_pow2(const uint32_t (&v)[16], int c0, uint32_t slot_local, int cnt,
-                                                  uint32_t recv_bar) {
-    constexpr int PER = 16 / SPLIT;                                  // rows per owner among 16 columns
-#pragma unroll
-    for (int o = 0; o < SPLIT; ++o) {
-        const uint32_t dst = map_to_rank(slot_local + (uint32_t)(c0 / SPLIT) * 4u, (uint32_t)o);
-        const uint32_t bar = map_to_rank(recv_bar, (uint32_t)o);
-        (void)cnt;
-        if (PER == 2) {
-            st_async_v2(dst, v[o], v[o + SPLIT], bar);
-        } else if (PER == 4) {
-            st_async_v4(dst, v[o], v[o + SPLIT], v[o + 2 * SPLIT], v[o + 3 * SPLIT], bar);
-        } else {   // PER == 8
-            st_async_v4(dst, v[o], v[o + SPLIT], v[o + 2 * SPLIT], v[o + 3 * SPLIT], bar);
-            st_async_v4(dst + 16, v[o + 4 * SPLIT], v[o + 5 * SPLIT], v[o + 6 * SPLIT], v[o + 7 * SPLIT], bar);
-        }
-    }
+    size_t ring = (size_t)stages * (kTileBytes + 256 * bn);
+    if (bn > 32 && ring < stream_push_bytes(bn, split)) ring = stream_push_bytes(bn, split);   // wide tiles receive into the ring
+    return ring + stream_recv_bytes(bn, split) + kPermRing * 512 + 512 + 1024;
 }
 
 template <int BN>
@@ -751,9 +739,14 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
     const int split = (int)gridDim.z, slice = (int)blockIdx.z;
-    // layout (matches stream_smem_bytes): stages | pushed partials | permutation ring | barriers
-    const uint32_t recv_off = (uint32_t)stages * L::kStage;
-    const uint32_t perm_off = recv_off + (split > 1 ? (uint32_t)L::kRecvBytes : 0u);
+    // layout (matches stream_smem_bytes): ring of stages | pushed partials (narrow tiles) | permutation ring | barriers;
+    // wide tiles receive the pushed partials at the start of the ring
+    const int cnt4 = stream_cnt4(BN, split);
+    const uint32_t push_bytes = split > 1 ? (uint32_t)(split * cnt4 * 512) : 0u;
+    uint32_t ring_bytes = (uint32_t)stages * L::kStage;
+    if (!L::kEarlyPush && ring_bytes < push_bytes) ring_bytes = push_bytes;
+    const uint32_t recv_off = L::kEarlyPush ? ring_bytes : 0u;
+    const uint32_t perm_off = ring_bytes + (L::kEarlyPush ? push_bytes : 0u);
     const uint32_t bar_off = perm_off + kPermRing * 512;
     const uint32_t bar_base = sbase + bar_off;
     auto full = [&](int s) { return bar_base + 8u * s; };
@@ -773,7 +766,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
     const int prefetch = min(stages, nk);
     const uint32_t rank = (split > 1) ? cluster_ctarank() : 0u;
-    const int cnt = (BN + split - 1) / split;                        // rows per owner (pitch of a feature's run in a slot)
+    const int owned = max(0, min(cnt4, BN - (int)rank * cnt4));      // rows of this tile that this CTA finishes
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(full(s), L::kProd + 1); mbar_init(empty(s), 1); }
@@ -781,11 +774,8 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
         mbar_init(recv_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
-        if (L::kPush && split > 1) {
-            // every sender delivers 128 features x (rows of this tile that this CTA owns) floats
-            const int owned = (BN - (int)rank + split - 1) / split;
-            mbar_arrive_expect_tx(recv_bar, (uint32_t)(split * owned * 512));
-        }
+        // every sender delivers 128 features x (rows of this tile that this CTA owns) floats
+        if (split > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)(split * owned * 512));
     }
     if (warp == 0) {
         // The weight stream starts now: nothing below is needed for these copies.  Lane s owns stage s (bulk copies
@@ -816,9 +806,14 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     if (split > 1) cluster_arrive();       // every CTA of the cluster is running and has its barriers set up
     grid_launch_dependents();
 
+    // Cluster barrier protocol (split > 1): phase A = "every CTA has its barriers set up" (arrived above); wide tiles add
+    // phase B = "every CTA's MMAs are done with the ring".  Every thread takes part in every phase, whatever happened to it.
     if (warp == 0) {
         // (later weight tiles are issued by the X producer warps below, right after they have seen the stage's `empty`)
-        if (split > 1) cluster_wait();
+        if (split > 1) {
+            cluster_wait();
+            if (!L::kEarlyPush) { cluster_arrive(); cluster_wait(); }
+        }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_sparse_f16(128, BN, 1);
@@ -845,7 +840,10 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
             tc_commit(accum_bar);
         }
         __syncwarp();
-        if (split > 1) cluster_wait();
+        if (split > 1) {
+            cluster_wait();
+            if (!L::kEarlyPush) { cluster_arrive(); cluster_wait(); }
+        }
     } else {
         // ---- X producers: thread g copies the 16-byte pieces e = g, g + 128, ... of the stage's 128 rows
         const int g = threadIdx.x - 64;
@@ -901,15 +899,16 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
                 bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
             }
         }
-        // ---- epilogue: the first four producer warps, one quarter of the accumulator lanes each
-        if (warp >= 6) {
-            if (split > 1) cluster_wait();
-        } else {
+        // ---- epilogue.  One K-slice: the first four producer warps (one quarter of the accumulator lanes each) stage
+        // the tile in shared memory and store it.  Several: every producer warp pushes partial rows to their owners
+        // (warp w reads lane quarter w % 4 and the 16-column pieces (w - 2) / 4, + kProd / 128, ...), then finishes the rows
+        // this CTA owns.
         const int quarter = warp & 3;
         const int f_local = quarter * 32 + lane;
-        const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
-        tc_fence_after();
         if (split == 1) {
+            if (warp < 6) {
+            const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
+            tc_fence_after();
             // accumulators -> shared memory [token][128 features] in the output type -> 16-byte stores
             const int esize = p.out_f32 ? 4 : 2;
             const float bias_f = epilogue_bias(p, (long)ft * 128 + f_local);
@@ -957,29 +956,17 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
                         }
                 }
             }
-        } else if (!L::kPush) {
-            // ---- stage the fp32 partial tile [token][128 features]; owners pull after the cluster barrier below
-            cluster_wait();
-            float *stage_f32 = reinterpret_cast<float *>(smem);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 16) {
-                uint32_t v[16];
-                if (nk > 0 && ok) {
-                    tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) v[e] = 0;
-                }
-#pragma unroll
-                for (int e = 0; e < 16; ++e) stage_f32[(c0 + e) * 128 + f_local] = __uint_as_float(v[e]);
             }
-            tc_fence_before();
         } else {
-            // ---- push the partial rows to their owners (row % split), then finish the rows this CTA owns
-            cluster_wait();                                          // all CTAs of the cluster have initialised their barriers
-            const uint32_t slot_local = sbase + recv_off + (uint32_t)(((int)rank * 128 + f_local) * cnt) * 4u;
+            constexpr int kPushGroups = L::kProd / 128;                  // 16-column pieces pushed side by side
+            const int cgrp = (warp - 2) >> 2;
+            const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
+            tc_fence_after();
+            cluster_wait();                                          // phase A: every CTA of the cluster has its barriers
+            if (!L::kEarlyPush) { cluster_arrive(); cluster_wait(); }   // phase B: every CTA's MMAs are done with the ring
+            const int groups = cnt4 >> 2;                            // 4-row groups per owner
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 16) {
+            for (int c0 = cgrp * 16; c0 < BN; c0 += 16 * kPushGroups) {
                 uint32_t v[16];
                 if (nk > 0 && ok) {
                     tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + c0, v);
@@ -987,67 +974,40 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
 #pragma unroll
                     for (int e = 0; e < 16; ++e) v[e] = 0;
                 }
-                if (split == 2) push_columns_pow2<2>(v, c0, slot_local, cnt, recv_bar);
-                else if (split == 4) push_columns_pow2<4>(v, c0, slot_local, cnt, recv_bar);
-                else if (split == 8) push_columns_pow2<8>(v, c0, slot_local, cnt, recv_bar);
-                else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int row = c0 + e;
-                        const uint32_t owner = (uint32_t)(row % split);
-                        st_async_b32(map_to_rank(slot_local + (uint32_t)(row / split) * 4u, owner), v[e],
-                                     map_to_rank(recv_bar, owner));
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    const int row = c0 + 4 * j;
+                    const int owner = row / cnt4, rg = (row - owner * cnt4) >> 2;
+                    const uint32_t local = sbase + recv_off + (uint32_t)((((int)rank * groups + rg) * 128 + f_local) * 16);
+                    st_async_v4(map_to_rank(local, (uint32_t)owner), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3],
+                                map_to_rank(recv_bar, (uint32_t)owner));
                 }
             }
             tc_fence_before();
             const bool got = mbar_wait_cluster(recv_bar, 0, abort_flag);
             const bool fine = got && (*abort_flag == 0);
-            const float *recv = reinterpret_cast<const float *>(smem + recv_off);
+            const float4 *recv = reinterpret_cast<const float4 *>(smem + recv_off);
             const int f_valid = min(128, p.N - ft * 128);
-            const int owned = (BN - (int)rank + split - 1) / split;
-            for (int q = g; q < owned * 128; q += 128) {
-                const int i = q >> 7, f = q & 127;
-                const int t = tok0 + i * split + (int)rank;
-                if (!fine || t >= p.M || f >= f_valid) continue;
-                float acc = 0.f;
-                for (int r = 0; r < split; ++r) acc += recv[(r * 128 + f) * cnt + i];   // slice order: deterministic
-                const long o = (long)t * p.ldy + (long)ft * 128 + f;
-                acc = epilogue_value(p, acc, (long)ft * 128 + f);
-                if (p.out_f32) reinterpret_cast<float *>(p.Y)[o] = acc;
-                else reinterpret_cast<__half *>(p.Y)[o] = __float2half_rn(acc);
+            for (int q = g; q < (owned >> 2) * 128; q += L::kProd) {
+                const int rg = q >> 7, f = q & 127;
+                float a[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int r = 0; r < split; ++r) {                    // slice order: deterministic
+                    const float4 part = recv[(r * groups + rg) * 128 + f];
+                    a[0] += part.x; a[1] += part.y; a[2] += part.z; a[3] += part.w;
+                }
+                if (!fine || f >= f_valid) continue;
+                const float bias_f = epilogue_bias(p, (long)ft * 128 + f);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int t = tok0 + (int)rank * cnt4 + rg * 4 + e;
+                    if (t >= p.M) continue;
+                    const long o = (long)t * p.ldy + (long)ft * 128 + f;
+                    const float y = epilogue_apply(a[e], bias_f, p.act);
+                    if (p.out_f32) reinterpret_cast<float *>(p.Y)[o] = y;
+                    else reinterpret_cast<__half *>(p.Y)[o] = __float2half_rn(y);
+                }
             }
         }
-        }
-    }
-    if (!L::kPush && split > 1) {
-        cluster_sync_all();                                          // every partial tile is staged
-        const bool fine = (*abort_flag == 0);
-        const int f_valid = min(128, p.N - ft * 128);
-        for (int q = threadIdx.x; q < BN * 32; q += L::kThreads) {            // 4 consecutive features of one row per thread
-            const int row = q >> 5, f0 = (q & 31) * 4;
-            if ((row % split) != (int)rank) continue;
-            const int t = tok0 + row;
-            if (t >= p.M || f0 >= f_valid) continue;
-            float4 part[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r)
-                if (r < split) part[r] = ld_dsmem_v4(sbase + (uint32_t)(row * 128 + f0) * 4u, (uint32_t)r);
-            float a[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int r = 0; r < 8; ++r)
-                if (r < split) { a[0] += part[r].x; a[1] += part[r].y; a[2] += part[r].z; a[3] += part[r].w; }   // slice order
-            if (fine) {
-                const long o = (long)t * p.ldy + (long)ft * 128 + f0;
-                for (int e = 0; e < 4; ++e)
-                    if (f0 + e < f_valid) {
-                        const float y = epilogue_value(p, a[e], (long)ft * 128 + f0 + e);
-                        if (p.out_f32) reinterpret_cast<float *>(p.Y)[o + e] = y;
-                        else reinterpret_cast<__half *>(p.Y)[o + e] = __float2half_rn(y);
-                    }
-            }
-        }
-        cluster_sync_all();                                          // nobody leaves while a peer still reads its tile
     }
     __syncthreads();
     if (warp == 1) {
@@ -1292,7 +1252,7 @@ static size_t ximg_bytes(int M, int K, int tn) {
 size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o) { return transpose_bytes(M, K, o); }
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
     size_t n = transpose_bytes(M, K, o);
-    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 1);
+    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 4);
     if (pair_possible) {
         size_t img = 0;
         for (int tn : {128, 192, 224, 240}) img = std::max(img, ximg_bytes(M, K, tn));
@@ -1341,20 +1301,23 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
         else if (o.force_kernel == ESP_KERNEL_PAIR_TILED) g.kernel = ESP_KERNEL_PAIR_TILED;
         else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
         else {
-            // The pair kernel (no K-slices) takes every M > 256, and 64 < M <= 256 when the weight has enough feature tiles
-            // to give it twenty clusters or more: there it beats the streaming kernel's gather and K-slice reduction
-            // (11008 x 4096 at 128 / 256 tokens: 33 against 47 / 51 us), below that it leaves most SMs idle.
-            const long clusters128 = (long)ceil_div(f_tiles, 4) * ceil_div(M, 128);
-            const bool pair = o.split_k <= 1 && (M > 256 || (M > 64 && clusters128 >= 20));
+            // The pair kernel takes every M > 64; a requested token tile or slice count that only the streaming kernel has
+            // (tiles below 128 tokens, more than four slices, slices of a 256-token tile) goes there.
+            const bool stream_only = (bn != 0 && bn < 128) || o.split_k > 4 || (bn == 256 && o.split_k > 1);
+            // Up to 256 tokens the pair kernel pays only where the weight gives it twenty pairs or more per K-slice (its
+            // set-up and drain cost about 10 us; measured at 128 tokens: 11008 x 4096 26.5 against the streaming kernel's
+            // 28.5 us, but 4096 x 4096 20.3 against 14.6).
+            const long pairs128 = (long)ceil_div(f_tiles, 4) * ceil_div(M, 128);
+            const bool pair = !stream_only && (M > 256 || (M > 64 && pairs128 >= 20));
             g.kernel = pair ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;
         }
     }
     if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED) {
+        const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
         if (bn == 0) {
             // cost ~ waves of clusters x time of one wave, in clocks: a channel step costs its MMAs (8 x TN/2 clocks) and its
             // 36 KB of weights + X tile (64-token blocks: 16 KB for TN = 128, else 32 KB) at the ~70 B/clk an SM pulls from
             // L2.  Wide tiles win once the grid fills the machine; a grid of less than one wave runs faster on narrow ones.
-            const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
             double best = -1.0;
             for (int tn : {240, 224, 192, 128}) {
                 const long clusters = f_pairs * ceil_div(M, tn);
@@ -1366,17 +1329,30 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
             }
         }
         if (bn != 128 && bn != 192 && bn != 224 && bn != 240 && bn != 256) return ESP_ERR_INVALID_ARG;
-        // the tiled form needs room for the X images behind the transposed copy; without it the gather form runs
+        // K-slices (128-token tiles only: the pushed partial rows of all slices must fit the ring): as many as fill one
+        // wave of pairs, each slice keeping at least four channel steps
+        int split = 1;
+        if (bn == 128) {
+            const long pairs = f_pairs * ceil_div(M, 128);
+            split = o.split_k > 0 ? o.split_k : (int)std::min<long>(4, std::max<long>(1, per_wave / pairs));
+            while (split > 1 && (k_tiles / split < 4 || (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles)) --split;
+        } else if (o.split_k > 1) {
+            return ESP_ERR_INVALID_ARG;
+        }
+        // the tiled form needs room for the X images behind the transposed copy; without it the gather form runs.  Up to
+        // 256 tokens the gather form is taken anyway: one launch instead of two, and X is small.
         const bool room = bn != 256 && workspace_bytes >= transpose_bytes(M, K, o) + ximg_bytes(M, K, bn);
         if (g.kernel == ESP_KERNEL_PAIR_TILED && !room) return ESP_ERR_WORKSPACE;
-        if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room) g.kernel = ESP_KERNEL_PAIR_TILED;
+        if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room && M > 256) g.kernel = ESP_KERNEL_PAIR_TILED;
         g.token_tile = bn;
-        g.split_k = 1;
+        g.split_k = split;
         g.stages = 0;
         *plan = g;
         return ESP_OK;
     }
-    if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    // (33..64 tokens: two 32-token tiles beat one of 64 unless the weight has many feature tiles -- the second pass over the
+    // weight comes from L2, and the narrow tile keeps more CTAs per SM; 5120 x 5120: 13.1 against 15.7 us)
+    if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? (f_tiles <= 64 && g.kernel == ESP_KERNEL_STREAM ? 32 : 64) : M <= 128 ? 128 : 256;
     if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
@@ -1414,11 +1390,13 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 if (cap <= 0) continue;
                 const long ctas = tiles * split;
                 const long waves = (ctas + cap - 1) / cap;
-                // (2, 4 or 8 slices push their partial rows as vectors; other counts go element by element: measured ~2 us slower)
-                const bool pow2 = (split & (split - 1)) == 0;
                 // per CTA: kts steps + set-up, reduction and epilogue, which grow with the token tile (measured: a 256-token
                 // tile in one wave of 32 steps beats three waves of 8)
-                double cost = (double)waves * (kts + 2.0 + bn / 32.0) + (split > 1 ? (pow2 ? 0.25 : 6.0) + 0.05 * split : 0.0) + 0.01 * r;
+                // wide token tiles are bound by their X gather, which CTAs sharing an SM share: a step costs as many
+                // times more as CTAs of one wave sit on an SM
+                const long in_wave = ctas < cap ? ctas : cap;
+                const double share = bn >= 64 ? (double)((in_wave + di.sm_count - 1) / di.sm_count) : 1.0;
+                double cost = (double)waves * (kts * share + 2.0 + bn / 32.0) + (split > 1 ? 0.25 + 0.05 * split : 0.0) + 0.01 * r;
                 // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
                 // (not when every CTA has an SM of its own anyway: a deeper ring is then free, measured 16.0 -> 12.6 us on
                 // 4096 x 4096 at 64 tokens)
@@ -1511,14 +1489,14 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             if (!p.x_channel_major) {        // token-major: one transposing tiling pass, no transposed copy
                 const uint16_t *xt = reinterpret_cast<const uint16_t *>(X);
                 switch (plan.token_tile) {
-                    case 128: st = launch_xtile_tm<128>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
+                    case 128: st = launch_xtile_tm<128>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream, plan.split_k);
                     case 192: st = launch_xtile_tm<192>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
                     case 224: st = launch_xtile_tm<224>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
                     default: st = launch_xtile_tm<240>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
                 }
             }
             switch (plan.token_tile) {
-                case 128: st = launch_xtile<128>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream);
+                case 128: st = launch_xtile<128>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream, plan.split_k);
                 case 192: st = launch_xtile<192>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 192, true>(p, true, stream);
                 case 224: st = launch_xtile<224>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 224, true>(p, true, stream);
                 default: st = launch_xtile<240>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 240, true>(p, true, stream);
@@ -1526,7 +1504,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
         }
         if (plan.kernel == ESP_KERNEL_PAIR) {
             switch (plan.token_tile) {
-                case 128: return launch_pair<2, 128>(p, dependent, stream);
+                case 128: return launch_pair<2, 128>(p, dependent, stream, plan.split_k);
                 case 192: return launch_pair<2, 192>(p, dependent, stream);
                 case 224: return launch_pair<2, 224>(p, dependent, stream);
                 case 240: return launch_pair<2, 240>(p, dependent, stream);

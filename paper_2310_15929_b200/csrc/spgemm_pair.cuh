@@ -304,11 +304,16 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     auto full = [&](int s) { return bar_base + 8u * s; };
     auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
     const uint32_t accum_bar = bar_base + 8u * 24;
+    const uint32_t recv_bar = bar_base + 8u * 26;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();                              // 0 = leader
+    // cluster (2, 1, split): ranks 2z and 2z + 1 are the CTA pair of K-slice z
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t rank = crank & 1u;                                     // 0 = leader of its pair
+    const uint32_t lead = crank & ~1u;                                    // cluster rank of the pair's leader
+    const int split = (int)gridDim.z, slice = (int)(crank >> 1);
     // Cluster -> tile.  Clusters start in the order of their linear index (x fastest).  Taken row by row, one wave of
     // clusters would span every feature pair on one or two token tiles, i.e. stream the whole weight from HBM once per
     // wave.  With p.raster_panel = P > 1 the index runs down panels of P token tiles instead (P tiles of one feature pair,
@@ -327,8 +332,11 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     }
     const int tok0 = ttile * TN;                                          // first token of the pair's tile
     const int tok_cta = tok0 + (int)rank * L::kHalf;                      // first token this CTA stages
-    const int nk = p.k_tiles;
+    const int kt_begin = slice * p.k_tiles_per_split;
+    const int nk = max(0, min(p.k_tiles, kt_begin + p.k_tiles_per_split) - kt_begin);
     const int f_tiles = (p.N + 127) / 128;
+    const int cnt4 = (((TN + split - 1) / split) + 3) & ~3;               // K-slice reduction: token rows per owner
+    const int owned = max(0, min(cnt4, TN - slice * cnt4));
     int ftile[NA];
     bool present[NA];
     int n_present = 0, n_present_peer = 0;
@@ -350,8 +358,11 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             mbar_init(empty(s), 1);
         }
         mbar_init(accum_bar, 1);
+        mbar_init(recv_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
+        // K-slices: every slice sends this CTA its owned rows of all NA accumulators (128 features x `owned` rows of fp32 each)
+        if (split > 1) mbar_arrive_expect_tx(recv_bar, (uint32_t)(NA * split * owned * 512));
     }
     if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), L::kTmemCols);
     // a feature tile beyond N: zero values and legal metadata once, never loaded
@@ -373,6 +384,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
 
     if (warp == 0) {
         // idle: keeps the producer warps at indices 2..17 (tensor-memory lane quarter = warp index % 4)
+        if (split > 1) cluster_sync_all();   // K-slices: "every pair's MMAs are done with the ring" (see the epilogue)
     } else if (warp == 1) {
         if (lane == 0 && rank != 0) {
             // gather form: forward "my operands of this stage have landed" to the leader
@@ -381,7 +393,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                 if (!mbar_wait_1t(full(s), ph, abort_flag)) break;
                 if (!TILED) fence_async_smem();   // rows written by cp.async (generic proxy) -> read by the MMA (async proxy)
-                mbar_arrive_remote(map_to_rank(full(s), 0));
+                mbar_arrive_remote(map_to_rank(full(s), lead));
             }
         } else if (lane == 0) {
             // One thread issues every MMA of the pair, so its own instruction stream must stay far shorter than the
@@ -389,6 +401,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // (>> 4) to their low words; the loop is unrolled over the ring and the metadata double buffer so that
             // every column index and offset is a compile-time constant.
             constexpr uint32_t idesc = instr_desc_sparse_f16(256, TN, 1);
+            const uint16_t pair_mask = (uint16_t)(3u << lead);            // both CTAs of this pair
             uint64_t ad0[NA][4], bd0[4], md0[NA];
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
@@ -432,12 +445,14 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                         }
                         if (it + 1 < nk) seen_b |= mbar_test(nbar, nph);
                     }
-                    tc_commit_pair(empty(s), (uint16_t)3);
+                    tc_commit_pair(empty(s), pair_mask);
                     seen = seen_a | seen_b;
                 }
             }
-            tc_commit_pair(accum_bar, (uint16_t)3);
+            tc_commit_pair(accum_bar, pair_mask);
         }
+        __syncwarp();
+        if (split > 1) cluster_sync_all();
     } else {
         const int g = threadIdx.x - 64;
         bool alive = true;
@@ -451,16 +466,16 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             if (lane == 0 && iw < kCopies * STAGES) {
                 const int s = iw / kCopies, kind = iw % kCopies;
                 const bool is_x = kind == NA;
-                const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * nk;
+                const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * p.k_tiles + kt_begin;
                 if (is_x || present[kind]) {
                     const uint32_t bytes = is_x ? (uint32_t)L::kXStage : (uint32_t)kTileBytes;
                     constexpr int kRowBytes = 1024;                       // the tensor maps see both buffers as 1024-byte rows
                     const CUtensorMap *map = is_x ? &xmap : &wmap;
-                    const int row0 = is_x ? (int)((ttile * 2 + rank) * nk) * (L::kXStage / kRowBytes)
-                                          : ftile[kind] * nk * (kTileBytes / kRowBytes);
+                    const int row0 = is_x ? (int)((ttile * 2 + rank) * p.k_tiles + kt_begin) * (L::kXStage / kRowBytes)
+                                          : (ftile[kind] * p.k_tiles + kt_begin) * (kTileBytes / kRowBytes);
                     const int row_step = (int)bytes / kRowBytes;
                     const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
-                    const uint32_t lead_full = map_to_rank(full(s), 0);
+                    const uint32_t lead_full = map_to_rank(full(s), lead);
                     for (int it = s; it < nk; it += STAGES) {
                         const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                         if (is_x) {
@@ -484,7 +499,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         const uint16_t *xb = reinterpret_cast<const uint16_t *>(p.X);
         constexpr int kAhead = 4;
         auto channel_of = [&](int it, int row) -> int {
-            const int kpos = it * kTileK + row;
+            const int kpos = (kt_begin + it) * kTileK + row;
             return (it < nk && kpos < p.K) ? (p.perm ? __ldg(p.perm + kpos) : kpos) : -1;
         };
         int nxt[kAhead][2];
@@ -528,7 +543,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                     if (present[a]) {
                         mbar_arrive_expect_tx(full(s), kTileBytes);
                         bulk_load(sbase + s * L::kStage + a * kTileBytes,
-                                  p.packed + ((long)ftile[a] * p.k_tiles + it) * kTileBytes, kTileBytes, full(s));
+                                  p.packed + ((long)ftile[a] * p.k_tiles + kt_begin + it) * kTileBytes, kTileBytes, full(s));
                     }
                 }
             }
@@ -594,7 +609,61 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 }
             }
         };
-        if (!p.out_f32) {
+        if (split > 1) {
+            // ---- K-slices: the pairs of the cluster hold partial sums of the same tile.  Its token rows are dealt to the
+            // slices in runs of cnt4 rows; every CTA sends, for each accumulator, the rows of each run to the CTA of the
+            // same pair rank in the owning slice (16-byte asynchronous remote stores: four token columns of one feature,
+            // completing on the owner's barrier), into the ring, which a cluster barrier has just declared free everywhere.
+            // The owner adds the slices in slice order and stores its rows.
+            cluster_sync_all();
+            const int groups = cnt4 >> 2;
+#pragma unroll 1
+            for (int a = 0; a < NA; ++a) {
+#pragma unroll 1
+                for (int c0 = cgrp * 16; c0 < TN; c0 += 64) {
+                    uint32_t v[16];
+                    if (nk > 0 && ok) {
+                        tmem_load_16(tmem + ((uint32_t)(quarter * 32) << 16) + L::acc_col(a) + c0, v);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) v[e] = 0;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int row = c0 + 4 * j;
+                        const int owner = row / cnt4, rg = (row - owner * cnt4) >> 2;
+                        const uint32_t local = sbase + (uint32_t)((((a * split + slice) * groups + rg) * 128 + f_local) * 16);
+                        const uint32_t dst_rank = (uint32_t)(2 * owner) + rank;
+                        st_async_v4(map_to_rank(local, dst_rank), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3],
+                                    map_to_rank(recv_bar, dst_rank));
+                    }
+                }
+            }
+            tc_fence_before();
+            const bool got = mbar_wait_cluster(recv_bar, 0, abort_flag);
+            const bool fine = got && ok && (*abort_flag == 0);
+            const float4 *recv = reinterpret_cast<const float4 *>(smem);
+            for (int q = g; q < NA * groups * 128; q += kPairProducers) {
+                const int a = q / (groups * 128), rg = (q / 128) % groups, f = q & 127;
+                if (rg * 4 >= owned || !present[a]) continue;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int z = 0; z < split; ++z) {                     // slice order: deterministic
+                    const float4 part = recv[((a * split + z) * groups + rg) * 128 + f];
+                    acc[0] += part.x; acc[1] += part.y; acc[2] += part.z; acc[3] += part.w;
+                }
+                const long feature = (long)ftile[a] * 128 + f;
+                if (!fine || feature >= p.N) continue;
+                const float bias_f = epilogue_bias(p, feature);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int t = tok0 + slice * cnt4 + rg * 4 + e;
+                    if (t >= p.M) continue;
+                    const float y = epilogue_apply(acc[e], bias_f, p.act);
+                    if (p.out_f32) reinterpret_cast<float *>(p.Y)[(long)t * p.ldy + feature] = y;
+                    else reinterpret_cast<__half *>(p.Y)[(long)t * p.ldy + feature] = __float2half_rn(y);
+                }
+            }
+        } else if (!p.out_f32) {
 #pragma unroll 1
             for (int a = 0; a < NA; ++a) stage_acc(a, smem + (size_t)a * TN * 256, __half());
             tc_fence_before();
@@ -693,13 +762,16 @@ inline esp_status_t make_rows_tensor_map(const void *base, size_t bytes, int box
 }
 
 template <int NA, int TN, bool TILED = false>
-esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream) {
+esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream, int split = 1) {
     using L = PairCfg<NA, TN>;
     auto kern = spgemm_pair_kernel<NA, TN, TILED>;
     ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
     const int f_tiles = (p.N + 127) / 128;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * ((f_tiles + 2 * NA - 1) / (2 * NA)), (p.M + TN - 1) / TN, 1);
+    // K-slices: the ring must hold the pushed partial rows of every slice (NA x split x cnt4 x 512 bytes)
+    const int cnt4 = (((TN + split - 1) / split) + 3) & ~3;
+    if (split < 1 || split > 4 || (split > 1 && (size_t)NA * split * cnt4 * 512 > (size_t)L::kStages * L::kStage)) return ESP_ERR_INVALID_ARG;
+    cfg.gridDim = dim3(2 * ((f_tiles + 2 * NA - 1) / (2 * NA)), (p.M + TN - 1) / TN, split);
     cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = L::kTotal;
     cfg.stream = stream;
@@ -707,7 +779,7 @@ esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t strea
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.z = split;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;

@@ -175,6 +175,39 @@ def test_pair_kernel_long_k_and_determinism():
     check(a, ref_product(X, vals, meta, theta), True)
 
 
+@pytest.mark.parametrize("kernel", [5, 6])
+@pytest.mark.parametrize("M,N,K", [(65, 640, 2048), (130, 200, 1160), (300, 384, 4224), (128, 512, 512)])
+def test_pair_kernel_k_slices(M, N, K, kernel):
+    """K-slices of the pair kernel (128-token tiles): the pairs of one cluster push their partial rows to the owning slice,
+    which adds them in slice order.  Every slice count against the oracle, both output types, with bias and ReLU applied to
+    the finished sum only; repeated calls give the same bits; the slices' sum order differs from the unsliced kernel's, so
+    the two are compared through the oracle, not with each other."""
+    from paper_2310_15929_b200 import binding as b
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(3 * M + N, N, K)
+    g = np.random.default_rng(M + K)
+    X = g.standard_normal((M, K)).astype(np.float16)
+    bias = (g.standard_normal(N) * 2).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Yref = ref_product(X, vals, meta, theta)
+    Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
+    for split in (2, 3, 4):
+        if K // 128 // split < 4:
+            continue                                              # the planner steps such a request down: covered by other counts
+        kw = dict(channel_major=True, kernel=kernel, token_tile=128, split_k=split)
+        a = spgemm(X, packed, theta, N, out_f32=True, **kw)
+        check(a, Yref, True)
+        assert np.array_equal(a, spgemm(X, packed, theta, N, out_f32=True, **kw))
+        check(spgemm(X, packed, theta, N, **kw), Yref)
+        check(spgemm(X, packed, theta, N, bias=bias, relu=True, **kw), Yb)
+        check(spgemm(X, packed, theta, N, kernel=kernel, token_tile=128, split_k=split), Yref)      # token-major X
+    o = b.esp_gemm_opts_default()
+    o.x_layout = b.ESP_X_CHANNEL_MAJOR
+    o.force_kernel, o.token_tile, o.split_k = kernel, 240, 2
+    with pytest.raises(b.EsparseError):                           # K-slices exist for 128-token tiles only
+        b.esp_spgemm_plan(M, N, K, o, True)
+
+
 def test_identity_permutation_and_unit_rows():
     """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
     from tests.gpu_util import pack_on_gpu, spgemm
