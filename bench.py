@@ -839,9 +839,17 @@ def main():
     ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "mid", "prune"],
                     help="run a few launches of one small case (for ncu) instead of the benchmark")
     ap.add_argument("--table5", action="store_true", help="time the GEMM shapes of the paper's Table 5 instead of the benchmark")
+    ap.add_argument("--per-config", default=None, metavar="W[,W...]",
+                    help="only the per-config sweep of these workloads (0..4), one JSON line per entry")
     args = ap.parse_args()
     if args.table5:
         run_table5(args)
+        return
+    if args.per_config is not None:
+        import torch
+        dev = torch.device("cuda", 0)
+        for e in per_config_sweep(dev, measured_peaks(), args.x_layout, only=[int(w) for w in args.per_config.split(",")]):
+            print(json.dumps(e), flush=True)
         return
     if args.profile_case:
         run_profile_case(args)

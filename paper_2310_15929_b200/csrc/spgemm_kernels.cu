@@ -1353,6 +1353,14 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
     // (33..64 tokens: two 32-token tiles beat one of 64 unless the weight has many feature tiles -- the second pass over the
     // weight comes from L2, and the narrow tile keeps more CTAs per SM; 5120 x 5120: 13.1 against 15.7 us)
     if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? (f_tiles <= 64 && g.kernel == ESP_KERNEL_STREAM ? 32 : 64) : M <= 128 ? 128 : 256;
+    // (a weight of a few tiles: narrow token tiles, so that the tiles x K-slices come to about one CTA per SM; re-reading
+    // so small a weight per token tile costs nothing.  512 x 512 at 128 tokens: 3.1 us with 16-token tiles against 8.4)
+    if (o.token_tile == 0 && g.kernel == ESP_KERNEL_STREAM && M > 16 && (long)f_tiles * k_tiles <= 64) {
+        for (int narrow : {16, 32, 64}) {
+            if (narrow >= bn) break;
+            if ((long)f_tiles * ceil_div(M, narrow) * std::min(k_tiles, 8) <= 2L * di.sm_count) { bn = narrow; break; }
+        }
+    }
     if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
