@@ -185,10 +185,13 @@ enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_PAIR = 5,      /* large M: two SMs share one 512-feature x token_tile MMA tile
                                     (token_tile 240 by default; 128, 192, 224 or 256 on request); X rows
                                     are gathered through the permutation by 16-byte copies              */
-       ESP_KERNEL_PAIR_TILED = 6 };/* the same tile, fed by bulk copies: a pass over X first writes the
+       ESP_KERNEL_PAIR_TILED = 6,/* the same tile, fed by bulk copies: a pass over X first writes the
                                     permuted, swizzled operand images into the workspace (default for
-                                    more than 256 tokens, and from 65 tokens on weights with many
-                                    feature tiles, when the workspace has room; token_tile 128..240)    */
+                                    more than 256 tokens when the workspace has room; token_tile 128..240) */
+       ESP_KERNEL_QUAD_TILED = 7 };/* ESP_KERNEL_PAIR_TILED with two such tiles (same features, neighbouring
+                                    token tiles) per cluster of four SMs: every weight tile is fetched once per
+                                    cluster and handed to the other pair through distributed shared memory
+                                    (token_tile 192, 224 or 240)                                        */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */

@@ -110,6 +110,20 @@ __device__ __forceinline__ bool mbar_wait_cluster_1t(uint32_t bar, uint32_t pari
     return mbar_wait_cluster(bar, parity, abort_flag);
 }
 
+// Tiled load of a [rows x 1024-byte] box into this CTA's shared memory, completing on one of this CTA's barriers.
+__device__ __forceinline__ void tma_rows_local(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                 "l"(map), "r"(0), "r"(row), "r"(bar)
+                 : "memory");
+}
+// Bulk copy from this CTA's shared memory into another CTA's of the cluster (plain peer copy, one source, one destination:
+// no multicast); the bytes complete on a barrier that lies in the destination CTA.
+__device__ __forceinline__ void dsmem_copy(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_cluster),
+                 "r"(src_cta), "r"(bytes), "r"(bar_cluster)
+                 : "memory");
+}
+
 constexpr int kPairProducers = 512;                  // X producer threads (warps 2..17)
 constexpr int kPairThreads = 64 + kPairProducers;
 
@@ -292,7 +306,7 @@ __device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *a
     return false;
 }
 
-template <int NA, int TN, bool TILED>
+template <int NA, int TN, bool TILED, bool QUAD = false>
 __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap wmap,
                                                                       const __grid_constant__ CUtensorMap xmap) {
     using L = PairCfg<NA, TN>;
@@ -305,24 +319,32 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     auto empty = [&](int s) { return bar_base + 8u * (8 + s); };
     const uint32_t accum_bar = bar_base + 8u * 24;
     const uint32_t recv_bar = bar_base + 8u * 26;
+    auto wland = [&](int s) { return bar_base + 8u * (16 + s); };     // QUAD: this CTA's own weight tile of the stage has landed
+    auto wrecv = [&](int s) { return bar_base + 8u * (32 + s); };     // QUAD: the partner's weight tile has arrived here
+    static_assert(!QUAD || (TILED && NA == 2), "the four-CTA form exists for the tiled two-accumulator kernel");
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // cluster (2, 1, split): ranks 2z and 2z + 1 are the CTA pair of K-slice z
+    // cluster (2, 1, split): ranks 2z and 2z + 1 are the CTA pair of K-slice z.
+    // QUAD, cluster (4, 1, 1): ranks 0, 1 and ranks 2, 3 are two pairs on the SAME 512 features and on neighbouring token
+    // tiles.  Each CTA fetches only one of its two weight tiles from L2 / HBM (the pair on the first token tile fetches
+    // accumulator 0's, the other pair accumulator 1's) and hands a copy to the CTA of the same pair rank in the other pair
+    // through distributed shared memory: a weight tile crosses the L2 -> SM path once per two token tiles.
     const uint32_t crank = cluster_ctarank();
     const uint32_t rank = crank & 1u;                                     // 0 = leader of its pair
     const uint32_t lead = crank & ~1u;                                    // cluster rank of the pair's leader
-    const int split = (int)gridDim.z, slice = (int)(crank >> 1);
+    const int split = QUAD ? 1 : (int)gridDim.z, slice = QUAD ? 0 : (int)(crank >> 1);
+    const int qpair = QUAD ? (int)(crank >> 1) : 0;                       // which of the cluster's two token tiles
     // Cluster -> tile.  Clusters start in the order of their linear index (x fastest).  Taken row by row, one wave of
     // clusters would span every feature pair on one or two token tiles, i.e. stream the whole weight from HBM once per
     // wave.  With p.raster_panel = P > 1 the index runs down panels of P token tiles instead (P tiles of one feature pair,
     // then the next pair): a wave then covers about 74 / P feature pairs x P token tiles, whose weight tiles and X images
     // together stay in L2 while the wave runs.
-    int pair_idx = (int)blockIdx.x >> 1;
-    int ttile = (int)blockIdx.y;
+    int pair_idx = (int)blockIdx.x >> (QUAD ? 2 : 1);
+    int ttile = (int)blockIdx.y;                                          // (QUAD: index of the pair of token tiles)
     if (p.raster_panel > 1) {
-        const int f_pairs = (int)gridDim.x >> 1, t_tiles = (int)gridDim.y;
+        const int f_pairs = (int)gridDim.x >> (QUAD ? 2 : 1), t_tiles = (int)gridDim.y;
         const int c = ttile * f_pairs + pair_idx;
         const int per_panel = p.raster_panel * f_pairs;
         const int panel = c / per_panel, r = c - panel * per_panel;
@@ -330,6 +352,8 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
         pair_idx = r / height;
         ttile = panel * p.raster_panel + (r - pair_idx * height);
     }
+    if (QUAD) ttile = 2 * ttile + qpair;
+    const bool has_tokens = ttile * TN < p.M;                             // (QUAD with an odd number of token tiles: the last cluster's second pair only hands on weights)
     const int tok0 = ttile * TN;                                          // first token of the pair's tile
     const int tok_cta = tok0 + (int)rank * L::kHalf;                      // first token this CTA stages
     const int kt_begin = slice * p.k_tiles_per_split;
@@ -353,9 +377,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // The MMA thread waits on one barrier per step, the leader's.  Gather form: one arrival per weight-tile copy +
             // the X threads, + rank 1's relayed "my stage has landed".  Tiled form: every copy of BOTH CTAs arrives on it
             // and reports its bytes to it directly (rank 1's own `full` barriers stay unused).
-            mbar_init(full(s), TILED ? 2u + (uint32_t)n_present + (uint32_t)n_present_peer
-                                     : (uint32_t)kPairProducers + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
-            mbar_init(empty(s), 1);
+            // QUAD: the X copies of both CTAs (if the pair has tokens) + from each CTA of the pair one "my own weight tile
+            // has landed" and one "the partner's tile has arrived"; a slot is free once BOTH pairs' MMAs are done with it.
+            mbar_init(full(s), QUAD ? (has_tokens ? 6u : 4u)
+                               : TILED ? 2u + (uint32_t)n_present + (uint32_t)n_present_peer
+                                       : (uint32_t)kPairProducers + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
+            mbar_init(empty(s), QUAD ? 2 : 1);
+            if (QUAD) { mbar_init(wland(s), 1); mbar_init(wrecv(s), 1); }
         }
         mbar_init(accum_bar, 1);
         mbar_init(recv_bar, 1);
@@ -445,7 +473,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                         }
                         if (it + 1 < nk) seen_b |= mbar_test(nbar, nph);
                     }
-                    tc_commit_pair(empty(s), pair_mask);
+                    tc_commit_pair(empty(s), QUAD ? (uint16_t)0xF : pair_mask);
                     seen = seen_a | seen_b;
                 }
             }
@@ -460,10 +488,72 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // ---- copy issuers: lane 0 of warp 2 + s * (NA + 1) + kind feeds ring slot s with weight tile `kind` (< NA) or
             // with the X image (kind == NA); it meets every phase of its slot's `empty` barrier.  The other lanes wait at
             // the vote below without polling.
-            constexpr int kCopies = NA + 1;
+            constexpr int kCopies = QUAD ? 4 : NA + 1;
             static_assert(kCopies * STAGES <= 15, "one issuing warp per copy of the ring; warp 17 polls the accumulator barrier");
             const int iw = warp - 2;
-            if (lane == 0 && iw < kCopies * STAGES) {
+            if (QUAD && lane == 0 && iw < kCopies * STAGES) {
+                // ---- four lanes per ring slot: 0 fetches this CTA's share of the weight tiles, 1 the X image, 2 hands the
+                // fetched tile on to the partner CTA once it has landed, 3 reports the tile received from the partner
+                const int s = iw / kCopies, role = iw % kCopies;
+                const int a_own = qpair, a_got = 1 - qpair;
+                const uint32_t partner = crank ^ 2u;
+                const uint32_t lead_full = map_to_rank(full(s), lead);
+                constexpr int kRowBytes = 1024;
+                if (role == 0) {
+                    const int row_step = kTileBytes / kRowBytes;
+                    const int row0 = ftile[a_own] * p.k_tiles * row_step;
+                    const uint32_t dst = sbase + s * L::kStage + a_own * kTileBytes;
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                        if (present[a_own]) {
+                            mbar_arrive_expect_tx(wland(s), kTileBytes);
+                            tma_rows_local(dst, &wmap, row0 + it * row_step, wland(s));
+                        } else {
+                            mbar_arrive(wland(s));
+                        }
+                    }
+                } else if (role == 1) {
+                    if (has_tokens) {
+                        const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * p.k_tiles;
+                        const int row_step = L::kXStage / kRowBytes;
+                        const int row0 = (int)((ttile * 2 + rank) * p.k_tiles) * row_step;
+                        const uint32_t dst = sbase + s * L::kStage + L::kWStage;
+                        for (int it = s; it < nk; it += STAGES) {
+                            const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                            if (!xflag_wait(xflag + it, abort_flag)) { alive = false; break; }
+                            asm volatile("fence.proxy.async;" ::: "memory");
+                            if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                            mbar_arrive_expect_tx_cluster(lead_full, (uint32_t)L::kXStage);
+                            tma_rows_pair(dst, &xmap, row0 + it * row_step, lead_full);
+                        }
+                    }
+                } else if (role == 2) {
+                    // (the partner's slot is free: this CTA's `empty` barrier of the round took both pairs' commits before
+                    // the tile was fetched)
+                    const uint32_t src = sbase + s * L::kStage + a_own * kTileBytes;
+                    const uint32_t dst = map_to_rank(src, partner), rbar = map_to_rank(wrecv(s), partner);
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!mbar_wait_1t(wland(s), ph, abort_flag)) { alive = false; break; }
+                        if (present[a_own]) {
+                            mbar_arrive_expect_tx_cluster(rbar, kTileBytes);
+                            dsmem_copy(dst, src, kTileBytes, rbar);
+                        } else {
+                            mbar_arrive_remote(rbar);
+                        }
+                        mbar_arrive_remote(lead_full);
+                    }
+                } else {
+                    (void)a_got;
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!mbar_wait_cluster_1t(wrecv(s), ph, abort_flag)) { alive = false; break; }
+                        mbar_arrive_remote(lead_full);
+                    }
+                }
+            }
+            if (!QUAD && lane == 0 && iw < kCopies * STAGES) {
                 const int s = iw / kCopies, kind = iw % kCopies;
                 const bool is_x = kind == NA;
                 const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * p.k_tiles + kt_begin;
@@ -792,6 +882,38 @@ esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t strea
         if (st == ESP_OK) st = make_rows_tensor_map(p.ximg, xtile_image_bytes<TN>(p.M, p.K), L::kXStage / 1024, &xmap);
         if (st != ESP_OK) return st;
     }
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, wmap, xmap));
+    return ESP_OK;
+}
+
+// The four-CTA form of the tiled pair kernel: two pairs per cluster on the same 512 features and two neighbouring token
+// tiles; each weight tile is fetched once per cluster and handed to the other pair through distributed shared memory.
+template <int TN>
+esp_status_t launch_quad(const GemmParams &p, bool dependent, cudaStream_t stream) {
+    using L = PairCfg<2, TN>;
+    auto kern = spgemm_pair_kernel<2, TN, true, true>;
+    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    const int f_tiles = (p.N + 127) / 128, t_tiles = (p.M + TN - 1) / TN;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(4 * ((f_tiles + 3) / 4), (t_tiles + 1) / 2, 1);
+    cfg.blockDim = dim3(kPairThreads);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 4;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    CUtensorMap wmap, xmap;
+    memset(&wmap, 0, sizeof(wmap));
+    memset(&xmap, 0, sizeof(xmap));
+    esp_status_t st = make_rows_tensor_map(p.packed, (size_t)f_tiles * p.k_tiles * kTileBytes, kTileBytes / 1024, &wmap);
+    if (st == ESP_OK) st = make_rows_tensor_map(p.ximg, xtile_image_bytes<TN>(p.M, p.K), L::kXStage / 1024, &xmap);
+    if (st != ESP_OK) return st;
     ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, p, wmap, xmap));
     return ESP_OK;
 }

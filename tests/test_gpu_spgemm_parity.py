@@ -208,6 +208,29 @@ def test_pair_kernel_k_slices(M, N, K, kernel):
         b.esp_spgemm_plan(M, N, K, o, True)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 200, 264), (520, 640, 1160), (1000, 1100, 520), (2048, 512, 4224)])
+def test_quad_kernel_shares_weight_tiles_between_two_pairs(M, N, K):
+    """The four-CTA form: two pairs of a cluster work on the same 512 features and neighbouring token tiles, each fetching
+    half of the weight tiles and handing them to the other through distributed shared memory.  Same MMAs in the same order
+    as the pair kernel, so the results must be identical bit for bit -- with an odd number of token tiles (the last
+    cluster's second pair only hands on weights), feature tiles beyond N, every token tile width, both layouts."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(M + N + K, N, K)
+    g = np.random.default_rng(M)
+    X = g.standard_normal((M, K)).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Yref = ref_product(X, vals, meta, theta)
+    for tile in (240, 224, 192):
+        a = spgemm(X, packed, theta, N, channel_major=True, kernel=7, token_tile=tile, out_f32=True)
+        check(a, Yref, True)
+        assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, kernel=6, token_tile=tile, out_f32=True))
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=7), Yref)
+    check(spgemm(X, packed, theta, N, kernel=7), Yref)                          # token-major X
+    bias = (g.standard_normal(N) * 2).astype(np.float16)
+    Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=7, bias=bias, relu=True, static_weights=1), Yb)
+
+
 def test_identity_permutation_and_unit_rows():
     """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
     from tests.gpu_util import pack_on_gpu, spgemm
