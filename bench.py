@@ -727,6 +727,8 @@ def run_profile_case(args):
         print(json.dumps({"case": case, "No": 1024, "C": K, "T": T, "ms": ms, "xcal_bytes": 2 * T * K}))
         return
     M = PREFILL_M if case == "prefill" else 128 if case == "mid" else DECODE_M
+    if args.profile_shape:
+        M, N, K = (int(v) for v in args.profile_shape.lower().split("x"))
     vals = (torch.randn(N, K // 2, device=dev) * 0.02).half()
     meta = torch.full((N, K // 8), 0xE4, dtype=torch.uint8, device=dev)
     packed = torch.empty(b.esp_packed_bytes(N, K), dtype=torch.uint8, device=dev)
@@ -838,6 +840,7 @@ def main():
     ap.add_argument("--quick", action="store_true", help="headline only: skip the decode, LLaMA-7B, per-config and producer sections")
     ap.add_argument("--profile-case", default=None, choices=["prefill", "decode", "mid", "prune"],
                     help="run a few launches of one small case (for ncu) instead of the benchmark")
+    ap.add_argument("--profile-shape", default=None, metavar="MxNxK", help="sizes of the prefill / decode / mid profile case")
     ap.add_argument("--table5", action="store_true", help="time the GEMM shapes of the paper's Table 5 instead of the benchmark")
     ap.add_argument("--per-config", default=None, metavar="W[,W...]",
                     help="only the per-config sweep of these workloads (0..4), one JSON line per entry")

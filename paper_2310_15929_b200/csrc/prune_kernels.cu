@@ -152,9 +152,20 @@ __global__ void calib_norm_kernel(int C, const double *__restrict__ sumsq, doubl
 // correctly rounded, which yields the exact bin for fp16 data.
 // grid (ceil(C/64), splits), block 256 = 8 channel-vectors of 8 x 32 token lanes; counters in shared memory.
 // --------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) histogram_kernel(const __half *__restrict__ X, int T, int C, long ldx,
-                                                        int rows_per_split, int bins, const double *__restrict__ lo,
-                                                        const double *__restrict__ hi, unsigned int *__restrict__ counts) {
+// The exact bin of one element (fp64), for the few elements the fp32 estimate cannot decide.  Kept out of line so that the
+// streaming loop carries none of its operands in registers: the channel's range is re-read (from L1) when needed.
+__device__ __noinline__ int histogram_exact_bin(float xf, int c, int bins, const double *__restrict__ lo,
+                                                const double *__restrict__ hi) {
+    const double l = lo[c];
+    const double rng = __dsub_rn(hi[c], l);
+    if (!(rng > 0.0)) return 0;                                          // a constant channel: everything in bin 0
+    const double q = __ddiv_rn(__dmul_rn(__dsub_rn((double)xf, l), (double)bins), rng);
+    return max(0, min(bins - 1, (int)floor(q)));                         // (the clamp at 0 only keeps a NaN in bounds)
+}
+
+__global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restrict__ X, int T, int C, long ldx,
+                                                           int rows_per_split, int bins, const double *__restrict__ lo,
+                                                           const double *__restrict__ hi, unsigned int *__restrict__ counts) {
     extern __shared__ unsigned int s_cnt[];   // [64][bins]
     for (int i = threadIdx.x; i < 64 * bins; i += 256) s_cnt[i] = 0;
     __syncthreads();
@@ -168,36 +179,36 @@ __global__ void __launch_bounds__(256) histogram_kernel(const __half *__restrict
         // exact in fp32 and r = K / (hi - lo) rounded once, q32 = (x - lo) * r is within 3 * 2^-24 relative of the exact
         // quotient, i.e. within K * 1.8e-7 absolute, so wherever q32 sits further than eps = K * 2^-21 from an integer its
         // floor IS the exact bin.  The elements that sit closer (about one in ten thousand, and always the channel's
-        // minimum and maximum) take the fp64 division.
-        double l[8], scale_den[8];
+        // minimum and maximum) take the fp64 division.  r = 0 sends every element of a channel there (a constant channel,
+        // or a range whose lower end is not an fp16 value).
         float lf[8], rf[8];
-        bool flat[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            l[k] = lo[c0 + k];
-            double rng = __dsub_rn(hi[c0 + k], l[k]);
-            flat[k] = !(rng > 0.0);
-            scale_den[k] = flat[k] ? 1.0 : rng;
-            lf[k] = (float)l[k];                                   // exact when the range is a channel's own (an fp16 value)
-            const bool lo_exact = (double)lf[k] == l[k];
-            rf[k] = (flat[k] || !lo_exact) ? 0.f : (float)((double)bins / rng);   // 0: every element takes the fp64 path
+            const double l = lo[c0 + k];
+            const double rng = __dsub_rn(hi[c0 + k], l);
+            lf[k] = (float)l;
+            rf[k] = (rng > 0.0 && (double)lf[k] == l) ? (float)((double)bins / rng) : 0.f;
         }
-        const double kb = (double)bins;
-        const float eps = (float)bins * 0x1p-21f;
-        auto count_row = [&](const uint4 &v) {
-            const __half *h = reinterpret_cast<const __half *>(&v);
+        // "further than eps from an integer" as one compare: |frac - 1/2| < 1/2 - eps
+        const float half_band = 0.5f - (float)bins * 0x1p-21f;
+        unsigned int *cnt_k[8];                                            // this thread's eight counter rows
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const float xf = __half2float(h[k]);
-                const float qf = (xf - lf[k]) * rf[k];
-                const float fl = floorf(qf);
-                const float fr = qf - fl;
-                int b = (int)fl;
-                if (!(fr > eps && fr < 1.f - eps)) {
-                    const double q = __ddiv_rn(__dmul_rn(__dsub_rn((double)xf, l[k]), kb), scale_den[k]);
-                    b = flat[k] ? 0 : max(0, min(bins - 1, (int)floor(q)));   // (the clamp at 0 only keeps a NaN in bounds)
+        for (int k = 0; k < 8; ++k) cnt_k[k] = s_cnt + (cl + k) * bins;
+        auto count_row = [&](const uint4 &v) {
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+            for (int k2 = 0; k2 < 4; ++k2) {
+                const float2 xf2 = __half22float2(h2[k2]);
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int k = 2 * k2 + e;
+                    const float xf = e ? xf2.y : xf2.x;
+                    const float qf = (xf - lf[k]) * rf[k];
+                    int b = __float2int_rd(qf);
+                    const float fr = qf - (float)b;
+                    if (!(fabsf(fr - 0.5f) < half_band)) b = histogram_exact_bin(xf, c0 + k, bins, lo, hi);
+                    atomicAdd(cnt_k[k] + b, 1u);
                 }
-                atomicAdd(&s_cnt[(cl + k) * bins + b], 1u);
             }
         };
         // four rows per thread in flight
