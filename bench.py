@@ -39,10 +39,12 @@ HEAD_WORKLOAD, HEAD_M = 3, 8192            # llama-65b-layer, prefill
 DECODE_WORKLOAD, DECODE_MS = 4, (1, 32)    # opt-66b-layer, decode
 SMALL_WORKLOAD, PREFILL_M, DECODE_M = 1, 2048, 16      # llama-7b-layer (what earlier runs of this benchmark timed)
 WORKLOAD = SMALL_WORKLOAD                  # the profile cases below run on this one
-# dram__bytes_read.sum + dram__bytes_write.sum of one GEMM launch, from the ncu captures summarised under profiles/
-# (None = the kernel has changed since the counters were taken)
-PREFILL_TRAFFIC_BYTES = None
-DECODE_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the GEMM launches of one step, from the one-pass ncu captures of the
+# full-size launches summarised under profiles/ (None = the kernel has changed since the counters were taken).
+# Headline step: 4 x (8192 x 8192) + 2 x (22016 x 8192) + (8192 x 22016) at 8192 tokens.
+PREFILL_TRAFFIC_BYTES = 4 * 0.906e9 + 2 * 2.13e9 + 2.23e9
+# Decode step at one token: 4 x (9216 x 9216) + (36864 x 9216) + (9216 x 36864).
+DECODE_TRAFFIC_BYTES = 4 * 98.4e6 + 386.1e6 + 387.4e6
 # bounded sample of the headline workload that the CPU oracle's product is timed on
 CPU_ROWS, CPU_FEATURES = 256, 1024
 
@@ -559,7 +561,7 @@ def run_ours(args):
             gms = graph_time(grouped_step, 10)
             dec[f"M={M}"] = {"ms_per_step": dms, "value": dgbs, "unit": "GB/s",
                              "roofline": {"bound": "hbm", "achieved": dgbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                          "frac": dgbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES,
+                                          "frac": dgbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES if M == 1 else None,
                                           "frac_of_nominal_8TBs": dgbs / 8000.0, "of": peaks["source"]},
                              "dense_cublas_ms_per_step": dense_dec_ms, "speedup_vs_dense": dense_dec_ms / dms,
                              "grouped_qkv": {"launches_per_layer": 4, "ms_per_step": gms, "value": dbytes / (gms * 1e-3) / 1e9,
@@ -734,7 +736,9 @@ def run_profile_case(args):
     packed = torch.empty(b.esp_packed_bytes(N, K), dtype=torch.uint8, device=dev)
     b.esp_pack(vals, meta, N, K, packed)
     perm = torch.randperm(K, device=dev).int()
-    X = torch.randn(K, M, device=dev).half()
+    Xc = torch.zeros(K, (M + 7) // 8 * 8, dtype=torch.float16, device=dev)      # leading dimension: a multiple of 8 elements
+    Xc[:, :M] = torch.randn(K, M, device=dev).half()
+    X = Xc[:, :M]
     Y = torch.empty(M, N, dtype=torch.float16, device=dev)
     o = b.esp_gemm_opts_default(); o.x_layout = b.ESP_X_CHANNEL_MAJOR
     nws = b.esp_spgemm_workspace_bytes(M, N, K, o)

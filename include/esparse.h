@@ -188,10 +188,15 @@ enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_PAIR_TILED = 6,/* the same tile, fed by bulk copies: a pass over X first writes the
                                     permuted, swizzled operand images into the workspace (default for
                                     more than 256 tokens when the workspace has room; token_tile 128..240) */
-       ESP_KERNEL_QUAD_TILED = 7 };/* ESP_KERNEL_PAIR_TILED with two such tiles (same features, neighbouring
+       ESP_KERNEL_QUAD_TILED = 7,/* ESP_KERNEL_PAIR_TILED with two such tiles (same features, neighbouring
                                     token tiles) per cluster of four SMs: every weight tile is fetched once per
                                     cluster and handed to the other pair through distributed shared memory
-                                    (token_tile 192, 224 or 240)                                        */
+                                    (token_tile 192, 224 or 240; slower than ESP_KERNEL_PAIR_TILED on every
+                                    shape measured: kept for comparison)                                */
+       ESP_KERNEL_PAIR_PERSIST = 8 };/* ESP_KERNEL_PAIR_TILED as a persistent kernel: one CTA pair per two SMs walks
+                                    the tiles, the operand ring never drains between tiles and the epilogue (warps of
+                                    its own, accumulators straight from registers to Y) runs under the next tile's
+                                    first steps (token_tile 192, 224 or 240; same results bit for bit)      */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */

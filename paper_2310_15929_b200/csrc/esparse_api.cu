@@ -47,7 +47,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
     if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
         o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR && o->force_kernel != ESP_KERNEL_PAIR_TILED &&
-        o->force_kernel != ESP_KERNEL_QUAD_TILED)
+        o->force_kernel != ESP_KERNEL_QUAD_TILED && o->force_kernel != ESP_KERNEL_PAIR_PERSIST)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->activation != ESP_ACT_NONE && o->activation != ESP_ACT_RELU) return ESP_ERR_INVALID_ARG;

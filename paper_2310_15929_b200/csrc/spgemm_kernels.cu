@@ -1126,6 +1126,7 @@ inline esp_status_t tensor_map_encoder(EncodeTiledFn *out) {
 }
 
 #include "spgemm_pair.cuh"
+#include "spgemm_persist.cuh"
 
 // Tensor map over channel-major X: dim 0 = tokens (contiguous), dim 1 = channels (ldx apart); box = 64 tokens
 // x 1 row (the row-gather form loads four such rows per instruction), 128-byte swizzle, zero fill outside.
@@ -1252,7 +1253,8 @@ static size_t ximg_bytes(int M, int K, int tn) {
 size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o) { return transpose_bytes(M, K, o); }
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
     size_t n = transpose_bytes(M, K, o);
-    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 4) || o.force_kernel == ESP_KERNEL_QUAD_TILED;
+    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 4) || o.force_kernel == ESP_KERNEL_QUAD_TILED ||
+                               o.force_kernel == ESP_KERNEL_PAIR_PERSIST;
     if (pair_possible) {
         size_t img = 0;
         for (int tn : {128, 192, 224, 240}) img = std::max(img, ximg_bytes(M, K, tn));
@@ -1300,6 +1302,7 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
         else if (o.force_kernel == ESP_KERNEL_PAIR) g.kernel = ESP_KERNEL_PAIR;
         else if (o.force_kernel == ESP_KERNEL_PAIR_TILED) g.kernel = ESP_KERNEL_PAIR_TILED;
         else if (o.force_kernel == ESP_KERNEL_QUAD_TILED) g.kernel = ESP_KERNEL_QUAD_TILED;
+        else if (o.force_kernel == ESP_KERNEL_PAIR_PERSIST) g.kernel = ESP_KERNEL_PAIR_PERSIST;
         else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
         else {
             // The pair kernel takes every M > 64; a requested token tile or slice count that only the streaming kernel has
@@ -1313,7 +1316,8 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
             g.kernel = pair ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;
         }
     }
-    if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED || g.kernel == ESP_KERNEL_QUAD_TILED) {
+    const bool wide_only = g.kernel == ESP_KERNEL_QUAD_TILED || g.kernel == ESP_KERNEL_PAIR_PERSIST;   // no 128-token form
+    if (g.kernel == ESP_KERNEL_PAIR || g.kernel == ESP_KERNEL_PAIR_TILED || wide_only) {
         const long f_pairs = ceil_div(f_tiles, 4), per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
         if (bn == 0) {
             // cost ~ waves of clusters x time of one wave, in clocks: a channel step costs its MMAs (8 x TN/2 clocks) and its
@@ -1321,7 +1325,7 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
             // L2.  Wide tiles win once the grid fills the machine; a grid of less than one wave runs faster on narrow ones.
             double best = -1.0;
             for (int tn : {240, 224, 192, 128}) {
-                if (tn == 128 && g.kernel == ESP_KERNEL_QUAD_TILED) continue;          // (no 128-token form of the four-CTA kernel)
+                if (tn == 128 && wide_only) continue;
                 const long clusters = f_pairs * ceil_div(M, tn);
                 const double mma = 4.0 * tn, copy = (36864.0 + (tn > 128 ? 32768.0 : 16384.0)) / 70.0;
                 // per wave: the channel steps (both terms show in the measured step time), an epilogue that grows with the
@@ -1344,8 +1348,8 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
         // the tiled form needs room for the X images behind the transposed copy; without it the gather form runs.  Up to
         // 256 tokens the gather form is taken anyway: one launch instead of two, and X is small.
         const bool room = bn != 256 && workspace_bytes >= transpose_bytes(M, K, o) + ximg_bytes(M, K, bn);
-        if ((g.kernel == ESP_KERNEL_PAIR_TILED || g.kernel == ESP_KERNEL_QUAD_TILED) && !room) return ESP_ERR_WORKSPACE;
-        if (g.kernel == ESP_KERNEL_QUAD_TILED && bn == 128) return ESP_ERR_INVALID_ARG;
+        if ((g.kernel == ESP_KERNEL_PAIR_TILED || wide_only) && !room) return ESP_ERR_WORKSPACE;
+        if (wide_only && (bn == 128 || bn == 256)) return ESP_ERR_INVALID_ARG;
         if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room && M > 256) g.kernel = ESP_KERNEL_PAIR_TILED;
         g.token_tile = bn;
         g.split_k = split;
@@ -1457,7 +1461,8 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
     p.xflags = nullptr;
     p.raster_panel = 0;
     const int f_tiles = ceil_div(N, kTileFeat), t_tiles = ceil_div(M, plan.token_tile);
-    if (plan.kernel == ESP_KERNEL_PAIR || plan.kernel == ESP_KERNEL_PAIR_TILED || plan.kernel == ESP_KERNEL_QUAD_TILED) {
+    if (plan.kernel == ESP_KERNEL_PAIR || plan.kernel == ESP_KERNEL_PAIR_TILED || plan.kernel == ESP_KERNEL_QUAD_TILED ||
+        plan.kernel == ESP_KERNEL_PAIR_PERSIST) {
         // Panels pay once a row of clusters (every feature pair on one token tile) is a good part of a wave: about eight
         // token tiles per panel (six where the weight has few feature pairs), the panels evened out over the token tiles.
         // Measured (M = 8192 unless noted): 22016 x 8192 1.79 -> 1.96 PFLOP/s; 36864 x 9216 at 4096 tokens 1.56 -> 1.94;
@@ -1482,8 +1487,12 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             p.x_channel_major = 1;
         }
         const bool dependent = o.static_weights != 0;
-        if (plan.kernel == ESP_KERNEL_PAIR_TILED || plan.kernel == ESP_KERNEL_QUAD_TILED) {
+        if (plan.kernel == ESP_KERNEL_PAIR_TILED || plan.kernel == ESP_KERNEL_QUAD_TILED || plan.kernel == ESP_KERNEL_PAIR_PERSIST) {
             const bool quad = plan.kernel == ESP_KERNEL_QUAD_TILED;
+            const bool persist = plan.kernel == ESP_KERNEL_PAIR_PERSIST;
+            DeviceInfo di;
+            if (device_info(&di) != ESP_OK) return ESP_ERR_CUDA;
+            const int sms = di.sm_count;
             const size_t off = transpose_bytes(M, K, o);
             if (!workspace || workspace_bytes < off + ximg_bytes(M, K, plan.token_tile)) return ESP_ERR_WORKSPACE;
             uint8_t *img = reinterpret_cast<uint8_t *>(workspace) + off;
@@ -1503,16 +1512,16 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
                 const uint16_t *xt = reinterpret_cast<const uint16_t *>(X);
                 switch (plan.token_tile) {
                     case 128: st = launch_xtile_tm<128>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream, plan.split_k);
-                    case 192: st = launch_xtile_tm<192>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<192>(p, true, stream) : launch_pair<2, 192, true>(p, true, stream);
-                    case 224: st = launch_xtile_tm<224>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<224>(p, true, stream) : launch_pair<2, 224, true>(p, true, stream);
-                    default: st = launch_xtile_tm<240>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<240>(p, true, stream) : launch_pair<2, 240, true>(p, true, stream);
+                    case 192: st = launch_xtile_tm<192>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<192>(p, true, stream) : persist ? launch_pair_persist<192>(p, true, stream, sms) : launch_pair<2, 192, true>(p, true, stream);
+                    case 224: st = launch_xtile_tm<224>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<224>(p, true, stream) : persist ? launch_pair_persist<224>(p, true, stream, sms) : launch_pair<2, 224, true>(p, true, stream);
+                    default: st = launch_xtile_tm<240>(p, xt, ldx, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<240>(p, true, stream) : persist ? launch_pair_persist<240>(p, true, stream, sms) : launch_pair<2, 240, true>(p, true, stream);
                 }
             }
             switch (plan.token_tile) {
                 case 128: st = launch_xtile<128>(p, img, flags, dependent, stream); return st != ESP_OK ? st : launch_pair<2, 128, true>(p, true, stream, plan.split_k);
-                case 192: st = launch_xtile<192>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<192>(p, true, stream) : launch_pair<2, 192, true>(p, true, stream);
-                case 224: st = launch_xtile<224>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<224>(p, true, stream) : launch_pair<2, 224, true>(p, true, stream);
-                default: st = launch_xtile<240>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<240>(p, true, stream) : launch_pair<2, 240, true>(p, true, stream);
+                case 192: st = launch_xtile<192>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<192>(p, true, stream) : persist ? launch_pair_persist<192>(p, true, stream, sms) : launch_pair<2, 192, true>(p, true, stream);
+                case 224: st = launch_xtile<224>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<224>(p, true, stream) : persist ? launch_pair_persist<224>(p, true, stream, sms) : launch_pair<2, 224, true>(p, true, stream);
+                default: st = launch_xtile<240>(p, img, flags, dependent, stream); return st != ESP_OK ? st : quad ? launch_quad<240>(p, true, stream) : persist ? launch_pair_persist<240>(p, true, stream, sms) : launch_pair<2, 240, true>(p, true, stream);
             }
         }
         if (plan.kernel == ESP_KERNEL_PAIR) {

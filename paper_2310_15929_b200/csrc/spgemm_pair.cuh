@@ -21,7 +21,9 @@
 //   * 16-byte asynchronous row copies deliver about 25 GB/s per SM from 128 threads, 44 from 256 and 60 from
 //     512, independent of how many stages are in flight, so sixteen warps gather X.
 //
-// grid (2 x feature-pair tiles, token tiles, 1), cluster (2,1,1), block 576.  In both CTAs:
+// grid (2 x feature-pair tiles, token tiles, K-slices), cluster (2, 1, K-slices), block 576 (one K-slice unless the planner
+// splits a 128-token grid that is far below one wave; the four-CTA form at the end of this comment uses cluster (4,1,1)).
+// In both CTAs of a pair:
 //   warp 0             idle
 //   warp 1             tensor-memory allocation; lane 0 of the leader CTA (rank 0): tcgen05.cp + MMAs for the pair;
 //                      lane 0 of rank 1: forwards "my stage is full" to the leader's barrier
@@ -36,6 +38,15 @@
 // lane 0 of a warp of its own; the sixteen warps no longer gather, they only run the epilogue.  The 16-byte gather
 // path delivers 32 B/clk per SM, bulk copies about 70: the price is one more pass over X.  That pass and the GEMM run
 // concurrently: the GEMM is launched as the pass's programmatic dependent and takes each image when its flag is up.
+//
+// K-slices (128-token tiles): the pairs of one cluster take consecutive ranges of channel steps; after a cluster barrier
+// every CTA pushes its fp32 partial rows to the CTA of the same pair rank in the owning slice (16-byte asynchronous remote
+// stores), which adds the slices in slice order.
+//
+// QUAD = true (tiled form only) puts two pairs on the same 512 features and neighbouring token tiles into one cluster of
+// four; each CTA fetches one of its two weight tiles and hands a copy to the other pair through distributed shared memory.
+// Correct and bit-identical to the plain form, but slower on every shape measured (the hand-over chain does not fit a
+// three-slot ring): kept for comparison, never planned.
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");

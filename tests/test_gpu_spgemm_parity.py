@@ -231,6 +231,31 @@ def test_quad_kernel_shares_weight_tiles_between_two_pairs(M, N, K):
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=7, bias=bias, relu=True, static_weights=1), Yb)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 200, 264), (520, 640, 1160), (1000, 1100, 520), (4100, 1536, 1160), (2048, 512, 4224)])
+def test_persistent_pair_kernel(M, N, K):
+    """The persistent form: one CTA pair per two SMs walks the tiles; ring slots, barrier phases and the metadata double
+    buffer run on across tiles, the epilogue warps write straight from registers while the next tile's MMAs start.  Same
+    MMAs in the same order as the plain tiled kernel: identical bits -- with more tiles than resident pairs (several tiles per
+    pair, a step count that is not a multiple of the ring depth), feature tiles beyond N, ragged M, both layouts."""
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(M + N + K + 1, N, K)
+    g = np.random.default_rng(M + 1)
+    X = g.standard_normal((M, K)).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Yref = ref_product(X, vals, meta, theta)
+    for tile in (240, 224, 192):
+        a = spgemm(X, packed, theta, N, channel_major=True, kernel=8, token_tile=tile, out_f32=True)
+        check(a, Yref, True)
+        assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, kernel=6, token_tile=tile, out_f32=True))
+    h = spgemm(X, packed, theta, N, channel_major=True, kernel=8)
+    check(h, Yref)
+    assert np.array_equal(h, spgemm(X, packed, theta, N, channel_major=True, kernel=6))
+    check(spgemm(X, packed, theta, N, kernel=8), Yref)                          # token-major X
+    bias = (g.standard_normal(N) * 2).astype(np.float16)
+    Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=8, bias=bias, relu=True, static_weights=1), Yb)
+
+
 def test_identity_permutation_and_unit_rows():
     """perm = NULL is the identity; unit-vector inputs read back rows of the pruned weight exactly."""
     from tests.gpu_util import pack_on_gpu, spgemm
