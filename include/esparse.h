@@ -196,7 +196,8 @@ enum { ESP_KERNEL_AUTO = 0,
        ESP_KERNEL_PAIR_PERSIST = 8 };/* ESP_KERNEL_PAIR_TILED as a persistent kernel: one CTA pair per two SMs walks
                                     the tiles, the operand ring never drains between tiles and the epilogue (warps of
                                     its own, accumulators straight from registers to Y) runs under the next tile's
-                                    first steps (token_tile 192, 224 or 240; same results bit for bit)      */
+                                    first steps (token_tile 192, 224 or 240; same results bit for bit; within a few
+                                    per cent of ESP_KERNEL_PAIR_TILED either way, so only esp_spgemm_tune picks it) */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */

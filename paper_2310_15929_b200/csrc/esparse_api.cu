@@ -320,6 +320,8 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
             }
         }
         cands.push_back({ESP_KERNEL_PAIR, 256, 1, 0});
+        if (M > 256)
+            for (int tile : {240, 224, 192}) cands.push_back({ESP_KERNEL_PAIR_PERSIST, tile, 1, 0});      // never planned, sometimes ahead
     }
     if (M <= 1024) {
         for (int tile : {16, 32, 64, 128, 256}) {

@@ -489,6 +489,12 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
     const int lane = threadIdx.x & 31;
     long long Ax = 0, D[4] = {0, 0, 0, 0};
     const uint16_t *col = Wt + (long)cx * ldt;
+    // The decision "is the candidate ahead of f2" is the fp64 comparison of |w_x| * s_x with |w_f2| * s_f2.  Its fp32 image
+    // (exact |w|, scores rounded once, one rounded multiply: each product within 2^-23 relative of its fp64 counterpart)
+    // decides it whenever the two products differ by more than 2^-21 of the larger: then the fp64 products differ the same
+    // way.  Only the rows that are closer (ties, zero padding) take the fp64 multiplies.
+    const float sx32 = (float)sx;
+    const float s32[4] = {(float)sc_fixed[0], (float)sc_fixed[1], (float)sc_fixed[2], (float)sc_fixed[3]};
     auto rows8 = [&](const uint4 &vx, long j) {
         const uint4 p0 = *reinterpret_cast<const uint4 *>(pk + j);
         const uint4 p1 = *reinterpret_cast<const uint4 *>(pk + j + 4);
@@ -498,10 +504,22 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
             const uint16_t hx = reinterpret_cast<const uint16_t *>(&vx)[e];
             const int f2 = (int)(pkv[e] >> 16);
             const uint16_t hf = (uint16_t)(pkv[e] & 0xFFFFu);
-            const double sf = f2 == 0 ? sc_fixed[0] : f2 == 1 ? sc_fixed[1] : f2 == 2 ? sc_fixed[2] : sc_fixed[3];
-            const double xx = __dmul_rn(half_bits_abs_to_double(hx), sx);
-            const double xf = __dmul_rn(half_bits_abs_to_double(hf), sf);
-            const bool kept = metric_ahead(xx, k, xf, f2);
+            const float px = __half2float(__ushort_as_half(hx)) * sx32;      // (hx, hf hold magnitudes: the sign bit is clear)
+            const float pf = __half2float(__ushort_as_half(hf)) * (f2 == 0 ? s32[0] : f2 == 1 ? s32[1] : f2 == 2 ? s32[2] : s32[3]);
+            const float big = fmaxf(fabsf(px), fabsf(pf));                 // (scores may be negative when the caller supplies them)
+            const float margin = big * 0x1p-21f;
+            const bool normal = big >= 0x1p-100f;                           // below, fp32 products lose relative accuracy
+            bool kept;
+            if (normal && px - pf > margin) {
+                kept = true;
+            } else if (normal && pf - px > margin) {
+                kept = false;
+            } else {
+                const double sf = f2 == 0 ? sc_fixed[0] : f2 == 1 ? sc_fixed[1] : f2 == 2 ? sc_fixed[2] : sc_fixed[3];
+                const double xx = __dmul_rn(half_bits_abs_to_double(hx), sx);
+                const double xf = __dmul_rn(half_bits_abs_to_double(hf), sf);
+                kept = metric_ahead(xx, k, xf, f2);
+            }
             const long long wf = kept ? half_bits_abs_fixed(hf) : 0;
             Ax += kept ? half_bits_abs_fixed(hx) : 0;
 #pragma unroll

@@ -23,6 +23,32 @@ namespace {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
 
+// Host-side caches of what a repeated call would otherwise redo (a decode call is a few microseconds of GPU time: the
+// host must not take longer).  All thread-local: no lock on the call path.
+//
+// The opt-in shared-memory size of a kernel sticks to the function: it is raised once per kernel, device and size.
+inline cudaError_t ensure_dynamic_smem(const void *kern, int bytes) {
+    struct Entry { const void *kern; int dev, bytes; };
+    thread_local Entry cache[96];
+    thread_local int n = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    for (int i = 0; i < n; ++i)
+        if (cache[i].kern == kern && cache[i].dev == dev) {
+            if (cache[i].bytes >= bytes) return cudaSuccess;
+            const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e == cudaSuccess) cache[i].bytes = bytes;
+            return e;
+        }
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && n < 96) cache[n++] = Entry{kern, dev, bytes};
+    return e;
+}
+inline bool log_plans() {
+    static const bool on = getenv("ESP_LOG") != nullptr;
+    return on;
+}
+
 struct GemmParams {
     const __half *X;
     long ldx;
@@ -398,7 +424,7 @@ template <int BN, int STAGES>
 esp_status_t launch_gather(const GemmParams &p, int f_tiles, int t_tiles, int split, cudaStream_t stream) {
     using L = GatherSmem<BN, STAGES>;
     auto kern = spgemm_gather_kernel<BN, STAGES>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, L::kTotal));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(f_tiles, t_tiles, split);
     cfg.blockDim = dim3(192);
@@ -1021,7 +1047,7 @@ esp_status_t launch_stream(const GemmParams &p, int f_tiles, int t_tiles, int sp
                            cudaStream_t stream) {
     auto kern = spgemm_stream_kernel<BN>;
     const size_t smem = stream_smem_bytes(BN, stages, split);
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, (int)smem));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(f_tiles, t_tiles, split);
     cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
@@ -1049,7 +1075,7 @@ template <int BN>
 esp_status_t launch_stream_group(const GemmGroup &grp, int t_tiles, int split, int stages, bool dependent, cudaStream_t stream) {
     auto kern = spgemm_stream_kernel<BN>;
     const size_t smem = stream_smem_bytes(BN, stages, split);
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, (int)smem));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grp.ft_start[grp.count], t_tiles, split);
     cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
@@ -1073,7 +1099,7 @@ template <int BN>
 int stream_cluster_capacity(int split, int stages) {
     auto kern = spgemm_stream_kernel<BN>;
     const size_t smem = stream_smem_bytes(BN, stages, split);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+    if (ensure_dynamic_smem((const void *)kern, (int)smem) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1, 1, split);
     cfg.blockDim = dim3(StreamCfg<BN>::kThreads);
@@ -1103,7 +1129,7 @@ int stream_cluster_capacity(int split, int stages) {
     per_sm = per_sm < 512 / (int)tmem_cols_for(BN) ? per_sm : 512 / (int)tmem_cols_for(BN);
     if (per_sm < api_per_sm) per_sm = api_per_sm;
     const int clusters = (int)((long)n * per_sm / api_per_sm);
-    if (getenv("ESP_LOG"))
+    if (log_plans())
         fprintf(stderr, "esparse occupancy tile=%d split=%d stages=%d smem=%zu: calculator clusters=%d at %d CTAs/SM, taken %d at %d CTAs/SM\n", BN,
                 split, stages, smem, n, api_per_sm, clusters, per_sm);
     return clusters;
@@ -1151,7 +1177,7 @@ esp_status_t launch_tma(const GemmParams &p, int f_tiles, int t_tiles, int split
     esp_status_t st = make_x_tensor_map(p.X, p.M, p.K, p.ldx, &map);
     if (st != ESP_OK) return st;
     auto kern = spgemm_tma_kernel<BN>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, L::kTotal));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(f_tiles, t_tiles, split);
     cfg.blockDim = dim3(192);
@@ -1286,7 +1312,7 @@ static int stream_capacity_ctas(int bn, int split, int stages) {
     return clusters * split;
 }
 
-esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan) {
+static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan) {
     const bool have_workspace = workspace_bytes >= transpose_bytes(M, K, o) && (workspace_bytes > 0 || o.x_layout == ESP_X_CHANNEL_MAJOR);
     DeviceInfo di;
     esp_status_t st = device_info(&di);
@@ -1418,7 +1444,7 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
                 if (o.static_weights && o.pipeline_stages == 0 && ctas > di.sm_count &&
                     2 * (stream_smem_bytes(bn, stages, split) + 1024) > (size_t)di.max_smem_optin)
                     cost += 3.0;
-                if (getenv("ESP_LOG"))
+                if (log_plans())
                     fprintf(stderr, "esparse plan M=%d N=%d K=%d tile=%d: split=%d stages=%d capacity=%d ctas=%ld waves=%ld cost=%.2f\n", M, N, K,
                             bn, split, stages, cap, ctas, waves, cost);
                 if (cost < best_cost) { best_cost = cost; best_split = split; best_stages = stages; }
@@ -1441,6 +1467,36 @@ esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t works
     g.split_k = split;
     *plan = g;
     return ESP_OK;
+}
+
+
+// The plan of a call is a pure function of its sizes, its options, the workspace size and the device: the last few are
+// remembered per thread, so that a layer's repeated calls do not walk the candidates again.
+esp_status_t plan_gemm(int M, int N, int K, const esp_gemm_opts &o, size_t workspace_bytes, GemmPlan *plan) {
+    struct Key { int dev, M, N, K, x_layout, split_k, force_kernel, token_tile, static_weights, pipeline_stages; size_t ws; };
+    struct Entry { Key key; GemmPlan plan; };
+    thread_local Entry cache[32];
+    thread_local int n = 0, next = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const Key key{dev, M, N, K, o.x_layout, o.split_k, o.force_kernel, o.token_tile, o.static_weights, o.pipeline_stages, workspace_bytes};
+    if (!log_plans())
+        for (int i = 0; i < n; ++i) {
+            const Key &k = cache[i].key;
+            if (k.dev == key.dev && k.M == key.M && k.N == key.N && k.K == key.K && k.x_layout == key.x_layout && k.split_k == key.split_k &&
+                k.force_kernel == key.force_kernel && k.token_tile == key.token_tile && k.static_weights == key.static_weights &&
+                k.pipeline_stages == key.pipeline_stages && k.ws == key.ws) {
+                *plan = cache[i].plan;
+                return ESP_OK;
+            }
+        }
+    const esp_status_t st = plan_gemm_uncached(M, N, K, o, workspace_bytes, plan);
+    if (st == ESP_OK) {
+        cache[next] = Entry{key, *plan};
+        next = (next + 1) % 32;
+        if (n < 32) ++n;
+    }
+    return st;
 }
 
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm, int N,

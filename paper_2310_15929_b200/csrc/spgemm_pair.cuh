@@ -458,10 +458,11 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
                 for (int u = 0; u < kUnroll; ++u) {
                     const int it = it0 + u;
                     if (it >= nk) break;
-                    const int s = u % STAGES;                             // == it % STAGES (it0 is a multiple of STAGES)
-                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    // it0 is a multiple of 2 * STAGES: slot and barrier phase of step it0 + u are compile-time constants
+                    const int s = u % STAGES;
+                    const uint32_t ph = (uint32_t)(u / STAGES) & 1u;
                     uint32_t seen_a = 0, seen_b = 0;
-                    const uint32_t nbar = full((u + 1) % STAGES), nph = (uint32_t)((it + 1) / STAGES) & 1u;
+                    const uint32_t nbar = full((u + 1) % STAGES), nph = (uint32_t)(((u + 1) % kUnroll) / STAGES) & 1u;
                     // Rank 1's arrival only relays that its stage is complete: one barrier for both CTAs, no cluster-scope
                     // acquire; a proxy fence only where the rows were written by cp.async.  A wait costs this thread ~300 clocks even
                     // when the phase is complete -- with the ~700 it needs to issue a step's MMAs that is more than the 960
@@ -849,6 +850,16 @@ esp_status_t launch_xtile(const GemmParams &p, uint8_t *img, uint32_t *flags, bo
 
 // Tensor map over a linear buffer seen as rows of 1024 bytes (256 32-bit words); box = box_rows whole rows, no swizzle.
 inline esp_status_t make_rows_tensor_map(const void *base, size_t bytes, int box_rows, CUtensorMap *map) {
+    // (a layer calls with the same buffers again and again: the last few maps are kept per thread)
+    struct Entry { const void *base; size_t bytes; int box_rows; CUtensorMap map; };
+    thread_local Entry cache[16];
+    thread_local int n = 0, next = 0;
+    for (int i = 0; i < n; ++i)
+        if (cache[i].base == base && cache[i].bytes == bytes && cache[i].box_rows == box_rows) {
+            *map = cache[i].map;
+            return ESP_OK;
+        }
+    Entry *slot = &cache[next];
     EncodeTiledFn encode = nullptr;
     esp_status_t st = tensor_map_encoder(&encode);
     if (st != ESP_OK) return st;
@@ -859,14 +870,18 @@ inline esp_status_t make_rows_tensor_map(const void *base, size_t bytes, int box
     CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? ESP_OK : ESP_ERR_CUDA;
+    if (r != CUDA_SUCCESS) return ESP_ERR_CUDA;
+    *slot = Entry{base, bytes, box_rows, *map};
+    next = (next + 1) % 16;
+    if (n < 16) ++n;
+    return ESP_OK;
 }
 
 template <int NA, int TN, bool TILED = false>
 esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t stream, int split = 1) {
     using L = PairCfg<NA, TN>;
     auto kern = spgemm_pair_kernel<NA, TN, TILED>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, L::kTotal));
     const int f_tiles = (p.N + 127) / 128;
     cudaLaunchConfig_t cfg = {};
     // K-slices: the ring must hold the pushed partial rows of every slice (NA x split x cnt4 x 512 bytes)
@@ -903,7 +918,7 @@ template <int TN>
 esp_status_t launch_quad(const GemmParams &p, bool dependent, cudaStream_t stream) {
     using L = PairCfg<2, TN>;
     auto kern = spgemm_pair_kernel<2, TN, true, true>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, L::kTotal));
     const int f_tiles = (p.N + 127) / 128, t_tiles = (p.M + TN - 1) / TN;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(4 * ((f_tiles + 3) / 4), (t_tiles + 1) / 2, 1);

@@ -13,14 +13,16 @@
 //     (barrier `acc_free`), not when their stores are done.
 // Same MMAs in the same order as the plain kernel: results are identical bit for bit.
 //
-// grid (2 x resident pairs), cluster (2,1,1), block 608:
-//   warp 0        idle (keeps tensor-memory lane quarter = warp index % 4 for the epilogue warps)
+// grid (2 x resident pairs), cluster (2,1,1), block 864:
+//   warp 0        idle
 //   warp 1        tensor-memory allocation; lane 0 of the leader CTA issues every tcgen05.cp / MMA of the pair
 //   warps 2..10   lane 0: copy issuer of ring slot (w - 2) / 3 for weight tile 0 / weight tile 1 / the X image
-//   warps 11..18  epilogue: warp w reads lane quarter w % 4; the 2 x TN/16 column pieces of a tile alternate between the
-//                 two warps of a quarter
-constexpr int kPersistEpiWarps = 8;
-constexpr int kPersistThreads = (2 + 9 + kPersistEpiWarps) * 32;
+//   warps 11..26  epilogue: warp w reads lane quarter w % 4 (a hardware rule); the 2 x TN/16 column pieces of a tile go
+//                 round the four warps of a quarter.  (Eight warps needed 7.7 us to read a tile's accumulators out, during
+//                 which the MMA thread waits: two warps per scheduler do not hide the load -> convert -> store chain.)
+constexpr int kPersistEpiWarps = 16;
+constexpr int kPersistFirstEpi = 11;
+constexpr int kPersistThreads = (kPersistFirstEpi + kPersistEpiWarps) * 32;
 
 template <int TN>
 __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel(const GemmParams p, const __grid_constant__ CUtensorMap wmap,
@@ -101,19 +103,21 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
 #pragma unroll
             for (int j = 0; j < 4; ++j) bd0[j] = smem_desc(sbase + L::kWStage + j * 4096, 16384, 1024, kLayoutSw128);
             constexpr int kUnroll = STAGES * 2;                           // ring slot and metadata buffer both periodic in the global step
-            const long total = (long)my_tiles * nk;
+            const int total = my_tiles * nk;
             bool alive = true;
             uint32_t seen = 0;
             int it = 0, tile_i = 0;
-            for (long gs0 = 0; gs0 < total && alive; gs0 += kUnroll) {
+            for (int gs0 = 0; gs0 < total && alive; gs0 += kUnroll) {
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    const long gs = gs0 + u;
+                    const int gs = gs0 + u;
                     if (gs >= total) break;
+                    // gs0 is a multiple of 2 * STAGES, so slot and barrier phase of step gs0 + u are compile-time constants
+                    // (this thread's instruction stream is the kernel's critical path: no division per step)
                     const int s = u % STAGES;
-                    const uint32_t ph = (uint32_t)(gs / STAGES) & 1u;
+                    const uint32_t ph = (uint32_t)(u / STAGES) & 1u;
                     uint32_t seen_a = 0, seen_b = 0;
-                    const uint32_t nbar = full((u + 1) % STAGES), nph = (uint32_t)((gs + 1) / STAGES) & 1u;
+                    const uint32_t nbar = full((u + 1) % STAGES), nph = (uint32_t)(((u + 1) % kUnroll) / STAGES) & 1u;
                     // a new tile overwrites the accumulators: the epilogue warps of both CTAs must have read the last one out
                     if (it == 0 && tile_i > 0 && !mbar_wait_cluster_1t(accfree_bar, (uint32_t)(tile_i - 1) & 1u, abort_flag)) { alive = false; break; }
                     if (!seen && !mbar_wait_1t(full(s), ph, abort_flag)) { alive = false; break; }
@@ -154,7 +158,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
             const int row_step = (int)bytes / kRowBytes;
             const uint32_t dst = sbase + s * L::kStage + (is_x ? L::kWStage : kind * kTileBytes);
             const uint32_t lead_full = map_to_rank(full(s), 0);
-            long base = 0;                                               // global step of the tile's first channel step
+            int base = 0;                                                // global step of the tile's first channel step
             bool alive = true;
             for (int c = cid; c < n_tiles && alive; c += n_clusters, base += nk) {
                 int pair_idx, ttile;
@@ -163,7 +167,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
                 const bool have = is_x || ft < f_tiles;
                 const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * nk;
                 const int row0 = is_x ? (int)((ttile * 2 + rank) * nk) * row_step : ft * nk * row_step;
-                for (int it = (int)(((s - base) % STAGES + STAGES) % STAGES); it < nk; it += STAGES) {
+                for (int it = ((s - base) % STAGES + STAGES) % STAGES; it < nk; it += STAGES) {
                     const uint32_t ph = (uint32_t)((base + it) / STAGES) & 1u;
                     if (is_x) {
                         if (!xflag_wait(xflag + it, abort_flag)) { alive = false; break; }
@@ -180,29 +184,31 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
             }
             if (!alive) *abort_flag = 1;
         }
-    } else if (warp >= 11) {
+    } else if (warp >= kPersistFirstEpi) {
         // ---- epilogue warps
         const int quarter = warp & 3;
-        const int half = (warp - 11) >> 2;                                // which of the quarter's two warps
-        const int f_local = quarter * 32 + lane;
+        const int sub = (warp - kPersistFirstEpi) >> 2;                   // which of the quarter's four warps
         constexpr int kPieces = TN / 16;                                  // 16-column pieces per accumulator
         const uint32_t lead_free = map_to_rank(accfree_bar, 0);
+        uint8_t *wbuf = smem + L::kBarOff + 512 + (size_t)(warp - kPersistFirstEpi) * 1024;   // this warp's transposition buffer (behind the barriers)
+        const bool y_vec = (reinterpret_cast<uintptr_t>(p.Y) & 15) == 0;
         int tile_i = 0;
         bool ok = true;
         for (int c = cid; c < n_tiles; c += n_clusters, ++tile_i) {
             int pair_idx, ttile;
             tile_of(c, pair_idx, ttile);
             const int tok0 = ttile * TN;
-            if (ok && nk > 0) {
-                bool got = true;
-                if (lane == 0) got = mbar_wait_cluster(accum_bar, (uint32_t)tile_i & 1u, abort_flag);
-                ok = __shfl_sync(0xFFFFFFFFu, (int)got, 0) != 0;
-            }
+            // one lane polls the accumulator barrier for all eight epilogue warps, which sleep on a named barrier meanwhile
+            // (lanes that poll through a whole main loop slow the CTA's other barrier operations down)
+            if (ok && nk > 0 && warp == kPersistFirstEpi && lane == 0 && !mbar_wait_cluster(accum_bar, (uint32_t)tile_i & 1u, abort_flag)) *abort_flag = 1;
+            __syncwarp();
+            asm volatile("bar.sync 1, %0;" ::"n"(kPersistEpiWarps * 32) : "memory");
+            ok = ok && *abort_flag == 0;
             tc_fence_after();
             int last_k = -1;
-            for (int k = half; k < NA * kPieces; k += 2) last_k = k;
+            for (int k = sub; k < NA * kPieces; k += 4) last_k = k;
 #pragma unroll 1
-            for (int k = half; k < NA * kPieces; k += 2) {
+            for (int k = sub; k < NA * kPieces; k += 4) {
                 const int a = k / kPieces, c0 = (k - a * kPieces) * 16;
                 uint32_t v[16];
                 if (nk > 0 && ok) {
@@ -217,23 +223,49 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
                     __syncwarp();
                     if (lane == 0) mbar_arrive_remote(lead_free);
                 }
+                // 16 tokens x this warp's 32 features: transposed through the warp's own 2 KB of shared memory, so that a lane
+                // stores 16 bytes of consecutive features of one token (sixteen 2-byte stores per lane, one feature each, made
+                // the epilogue several microseconds longer per tile)
                 const int ft = pair_idx * (2 * NA) + 2 * a + (int)rank;
-                const long feature = (long)ft * 128 + f_local;
-                if (!ok || ft >= f_tiles || feature >= p.N) continue;
-                const float bias_f = epilogue_bias(p, feature);
-                if (p.out_f32) {
-                    float *yo = reinterpret_cast<float *>(p.Y) + feature;
+                const long feat0 = (long)ft * 128 + quarter * 32;            // first feature of this warp's 32
+                const bool any = ok && ft < f_tiles && feat0 < p.N;
+                const float bias_f = any ? epilogue_bias(p, feat0 + lane) : 0.f;
+                const int esize = p.out_f32 ? 4 : 2;
+                const int per = 16 / esize;                                  // features per 16-byte piece
+                const int pieces_per_row = 32 / per;                         // 4 (fp16) or 8 (fp32)
+                const bool vec_ok = y_vec && (((long)p.ldy * esize) % 16 == 0);
+                // the buffer holds 1 KB: sixteen tokens of fp16, or eight of fp32 (two rounds)
+                const int rounds = p.out_f32 ? 2 : 1, tok_per_round = 16 / rounds;
+                for (int rd = 0; rd < rounds; ++rd) {
+                    __syncwarp();                                            // the previous piece has been read out of the buffer
+                    if (p.out_f32) {
+                        float *buf = reinterpret_cast<float *>(wbuf);
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int t = tok0 + c0 + e;
-                        if (t < p.M) yo[(long)t * p.ldy] = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
+                        for (int e = 0; e < 16; ++e)
+                            if ((e >> 3) == rd) buf[(e & 7) * 32 + lane] = epilogue_apply(__uint_as_float(v[e]), bias_f, p.act);
+                    } else {
+                        __half *buf = reinterpret_cast<__half *>(wbuf);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) buf[e * 32 + lane] = __float2half_rn(epilogue_apply(__uint_as_float(v[e]), bias_f, p.act));
                     }
-                } else {
-                    __half *yo = reinterpret_cast<__half *>(p.Y) + feature;
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int t = tok0 + c0 + e;
-                        if (t < p.M) yo[(long)t * p.ldy] = __float2half_rn(epilogue_apply(__uint_as_float(v[e]), bias_f, p.act));
+                    __syncwarp();
+                    if (!any) continue;
+                    for (int q = lane; q < tok_per_round * pieces_per_row; q += 32) {
+                        const int e = q / pieces_per_row, part = q % pieces_per_row;
+                        const int t = tok0 + c0 + rd * tok_per_round + e;
+                        if (t >= p.M) continue;
+                        const long f0 = feat0 + part * per;
+                        const uint8_t *src = wbuf + (size_t)(e * 32 + part * per) * esize;
+                        uint8_t *dstp = reinterpret_cast<uint8_t *>(p.Y) + ((long)t * p.ldy + f0) * esize;
+                        if (vec_ok && f0 + per <= p.N) {
+                            *reinterpret_cast<uint4 *>(dstp) = *reinterpret_cast<const uint4 *>(src);
+                        } else {
+                            for (int i = 0; i < per; ++i)
+                                if (f0 + i < p.N) {
+                                    if (p.out_f32) reinterpret_cast<float *>(dstp)[i] = reinterpret_cast<const float *>(src)[i];
+                                    else reinterpret_cast<uint16_t *>(dstp)[i] = reinterpret_cast<const uint16_t *>(src)[i];
+                                }
+                        }
                     }
                 }
             }
@@ -251,8 +283,10 @@ __global__ void __launch_bounds__(kPersistThreads, 1) spgemm_pair_persist_kernel
 template <int TN>
 esp_status_t launch_pair_persist(const GemmParams &p, bool dependent, cudaStream_t stream, int sm_count) {
     using L = PairCfg<2, TN>;
+    constexpr int kSmem = L::kTotal + kPersistEpiWarps * 1024;           // + the epilogue warps' transposition buffers
+    static_assert(kSmem <= 227 * 1024, "shared memory");
     auto kern = spgemm_pair_persist_kernel<TN>;
-    ESP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, kSmem));
     const int f_tiles = (p.N + 127) / 128, f_pairs = (f_tiles + 3) / 4, t_tiles = (p.M + TN - 1) / TN;
     const long n_tiles = (long)f_pairs * t_tiles;
     const int resident = sm_count / 2 > 0 ? sm_count / 2 : 1;            // one CTA per SM (tensor memory and shared memory are full)
@@ -260,7 +294,7 @@ esp_status_t launch_pair_persist(const GemmParams &p, bool dependent, cudaStream
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.blockDim = dim3(kPersistThreads);
-    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.dynamicSmemBytes = kSmem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -247,9 +247,10 @@ def test_persistent_pair_kernel(M, N, K):
         a = spgemm(X, packed, theta, N, channel_major=True, kernel=8, token_tile=tile, out_f32=True)
         check(a, Yref, True)
         assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, kernel=6, token_tile=tile, out_f32=True))
-    h = spgemm(X, packed, theta, N, channel_major=True, kernel=8)
+    h = spgemm(X, packed, theta, N, channel_major=True, kernel=8, token_tile=240)
     check(h, Yref)
-    assert np.array_equal(h, spgemm(X, packed, theta, N, channel_major=True, kernel=6))
+    assert np.array_equal(h, spgemm(X, packed, theta, N, channel_major=True, kernel=6, token_tile=240))
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=8), Yref)      # the planner's own tile
     check(spgemm(X, packed, theta, N, kernel=8), Yref)                          # token-major X
     bias = (g.standard_normal(N) * 2).astype(np.float16)
     Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
