@@ -193,11 +193,18 @@ enum { ESP_KERNEL_AUTO = 0,
                                     cluster and handed to the other pair through distributed shared memory
                                     (token_tile 192, 224 or 240; slower than ESP_KERNEL_PAIR_TILED on every
                                     shape measured: kept for comparison)                                */
-       ESP_KERNEL_PAIR_PERSIST = 8 };/* ESP_KERNEL_PAIR_TILED as a persistent kernel: one CTA pair per two SMs walks
+       ESP_KERNEL_PAIR_PERSIST = 8,/* ESP_KERNEL_PAIR_TILED as a persistent kernel: one CTA pair per two SMs walks
                                     the tiles, the operand ring never drains between tiles and the epilogue (warps of
                                     its own, accumulators straight from registers to Y) runs under the next tile's
                                     first steps (token_tile 192, 224 or 240; same results bit for bit; within a few
                                     per cent of ESP_KERNEL_PAIR_TILED either way, so only esp_spgemm_tune picks it) */
+       ESP_KERNEL_QUAD_MULTICAST = 9 };/* the cluster of ESP_KERNEL_QUAD_TILED with every weight tile delivered to
+                                    both pairs by ONE tiled load (cluster multicast of the tensor memory unit) instead
+                                    of a hand-over: token_tile 192, 224 or 240, same results bit for bit.  Its kernel
+                                    is in the optional companion library libesparse_mc.so, looked for beside this
+                                    library; without it the call returns ESP_ERR_UNSUPPORTED
+                                    (esp_multicast_available() tells).  Single-GPU use only: the packed weight must
+                                    lie in the memory of the GPU the call runs on.                      */
 
 typedef struct {
     size_t struct_size;          /* = sizeof(esp_gemm_opts)                                           */
@@ -333,6 +340,12 @@ esp_status_t esp_selftest_wait_timeout(void *cuda_stream);
  * kernel exits cleanly.  Returns ESP_OK if no kernel reported anything.
  */
 esp_status_t esp_last_device_status(void);
+
+/*
+ * 1 if the companion library with ESP_KERNEL_QUAD_MULTICAST was found beside this one and loaded, else 0 (no counterpart
+ * in the paper).  Host-only; the first call does the look-up.
+ */
+int esp_multicast_available(void);
 
 #ifdef __cplusplus
 }

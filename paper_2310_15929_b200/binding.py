@@ -20,7 +20,7 @@ ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
 ESP_ACT_NONE, ESP_ACT_RELU = 0, 1
 ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR, ESP_KERNEL_PAIR_TILED = 0, 1, 2, 4, 5, 6
-ESP_KERNEL_QUAD_TILED, ESP_KERNEL_PAIR_PERSIST = 7, 8
+ESP_KERNEL_QUAD_TILED, ESP_KERNEL_PAIR_PERSIST, ESP_KERNEL_QUAD_MULTICAST = 7, 8, 9
 
 
 class esp_prune_opts(ctypes.Structure):
@@ -57,7 +57,8 @@ EXPORTS = ("esp_status_string", "esp_version", "esp_prune_opts_default", "esp_ge
            "esp_metric_prune_workspace_bytes", "esp_packed_bytes", "esp_metric_prune", "esp_pack",
            "esp_decompress", "esp_spgemm_workspace_bytes", "esp_spgemm", "esp_last_device_status",
            "esp_spgemm_static", "esp_spgemm_plan", "esp_selftest_wait_timeout", "esp_calib_state_bytes", "esp_calib_reset",
-           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish", "esp_spgemm_tune", "esp_spgemm_grouped")
+           "esp_calib_range", "esp_calib_histogram", "esp_calib_finish", "esp_spgemm_tune", "esp_spgemm_grouped",
+           "esp_multicast_available")
 
 _lib.esp_status_string.restype = c_char_p
 _lib.esp_status_string.argtypes = [c_int]
@@ -82,6 +83,7 @@ _lib.esp_spgemm.restype = c_int
 _lib.esp_spgemm.argtypes = [c_void_p, c_int, c_int, c_long, c_void_p, c_void_p, c_int, c_void_p, c_long,
                             POINTER(esp_gemm_opts), c_void_p, c_size_t, c_void_p]
 _lib.esp_last_device_status.restype = c_int
+_lib.esp_multicast_available.restype = c_int
 _lib.esp_selftest_wait_timeout.restype = c_int
 _lib.esp_selftest_wait_timeout.argtypes = [c_void_p]
 _lib.esp_spgemm_plan.restype = c_int
@@ -348,3 +350,8 @@ def esp_calib_finish(state, C, T_total, opts, chan_norm, chan_entropy, chan_scor
 
 def esp_last_device_status() -> int:
     return int(_lib.esp_last_device_status())
+
+
+def esp_multicast_available() -> bool:
+    """True when the optional companion library (ESP_KERNEL_QUAD_MULTICAST) lies beside the main one and loads."""
+    return bool(_lib.esp_multicast_available())

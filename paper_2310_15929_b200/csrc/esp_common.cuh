@@ -81,7 +81,7 @@ esp_status_t launch_calib_finish(const CalibState &c, int C, int bins, long long
 
 // ---- GEMM launchers (spgemm_kernels.cu) ------------------------------------------------------------
 struct GemmPlan {
-    int kernel;        // ESP_KERNEL_GATHER | ESP_KERNEL_TMA | ESP_KERNEL_STREAM | ESP_KERNEL_PAIR | ESP_KERNEL_PAIR_TILED
+    int kernel;        // ESP_KERNEL_* (never AUTO)
     int token_tile;    // MMA N
     int split_k;       // cluster size along K
     int stages;
@@ -94,6 +94,9 @@ esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, 
                                  const int32_t *const *perm, const int *N, void *const *Y, const long *ldy,
                                  const esp_gemm_opts &o, void *workspace, size_t workspace_bytes, cudaStream_t stream);
 esp_status_t launch_wait_timeout_selftest(cudaStream_t stream);
+// The optional companion library (ESP_KERNEL_QUAD_MULTICAST): found and loaded?  Its device status word (0 if absent).
+bool companion_available();
+esp_status_t companion_device_status(int *out);
 esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *packed, const int32_t *perm,
                            int N, void *Y, long ldy, const esp_gemm_opts &o, const GemmPlan &plan,
                            void *workspace, size_t workspace_bytes, cudaStream_t stream);

@@ -47,7 +47,8 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->split_k < 0 || o->split_k > 8) return ESP_ERR_INVALID_ARG;
     if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
         o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR && o->force_kernel != ESP_KERNEL_PAIR_TILED &&
-        o->force_kernel != ESP_KERNEL_QUAD_TILED && o->force_kernel != ESP_KERNEL_PAIR_PERSIST)
+        o->force_kernel != ESP_KERNEL_QUAD_TILED && o->force_kernel != ESP_KERNEL_PAIR_PERSIST &&
+        o->force_kernel != ESP_KERNEL_QUAD_MULTICAST)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->activation != ESP_ACT_NONE && o->activation != ESP_ACT_RELU) return ESP_ERR_INVALID_ARG;
@@ -388,7 +389,11 @@ esp_status_t esp_last_device_status(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return ESP_ERR_CUDA;
     if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return ESP_ERR_CUDA;
     if (h != 0 && cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return ESP_ERR_CUDA;
-    return (esp_status_t)h;
+    int hc = 0;                               // the companion library's kernels have a status word of their own
+    if (companion_device_status(&hc) != ESP_OK) return ESP_ERR_CUDA;
+    return (esp_status_t)(h != 0 ? h : hc);
 }
+
+int esp_multicast_available(void) { return companion_available() ? 1 : 0; }
 
 }  // extern "C"

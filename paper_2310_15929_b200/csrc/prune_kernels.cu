@@ -163,11 +163,19 @@ __device__ __noinline__ int histogram_exact_bin(float xf, int c, int bins, const
     return max(0, min(bins - 1, (int)floor(q)));                         // (the clamp at 0 only keeps a NaN in bounds)
 }
 
+// Counters in shared memory: [k = channel within the thread's eight][bin][tx = the thread's channel group][replica].
+// The 32 lanes of a warp are 8 channel groups x 4 token rows, and one instruction counts the same k in all of them, so a
+// lane's bank is (bin * 8 + tx) * R + replica: lanes of different channel groups never meet in a bank, and the four lanes
+// of a group meet only through the low bits of their bins.  R = 4 gives each of them a counter row of its own (no conflict
+// at all), R = 2 one per two, R = 1 none (expected 1.0 / 1.5 / 2.1 passes per counting instruction; the plain
+// [channel][bin] layout needed 3.3).  R is chosen so that three CTAs still fit an SM.
+constexpr int kHistAhead = 8;                 // rows each thread keeps in flight
+template <int R>
 __global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restrict__ X, int T, int C, long ldx,
                                                            int rows_per_split, int bins, const double *__restrict__ lo,
                                                            const double *__restrict__ hi, unsigned int *__restrict__ counts) {
-    extern __shared__ unsigned int s_cnt[];   // [64][bins]
-    for (int i = threadIdx.x; i < 64 * bins; i += 256) s_cnt[i] = 0;
+    extern __shared__ __align__(16) unsigned int s_cnt[];   // [8][bins][8][R] | the threads' load rings: [kHistAhead + 1][256] x 16 bytes
+    for (int i = threadIdx.x; i < 64 * R * bins; i += 256) s_cnt[i] = 0;
     __syncthreads();
     const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;
     const int cl = tx * 8;
@@ -175,25 +183,32 @@ __global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restr
     const int r_begin = blockIdx.y * rows_per_split;
     const int r_end = min(T, r_begin + rows_per_split);
     if (c0 < C) {
-        // Exact bin: floor of the fp64 quotient (x - lo) * K / (hi - lo).  Almost every element gets there in fp32: with lo
-        // exact in fp32 and r = K / (hi - lo) rounded once, q32 = (x - lo) * r is within 3 * 2^-24 relative of the exact
-        // quotient, i.e. within K * 1.8e-7 absolute, so wherever q32 sits further than eps = K * 2^-21 from an integer its
-        // floor IS the exact bin.  The elements that sit closer (about one in ten thousand, and always the channel's
-        // minimum and maximum) take the fp64 division.  r = 0 sends every element of a channel there (a constant channel,
-        // or a range whose lower end is not an fp16 value).
+        // Exact bin: floor of the fp64 quotient q = (x - lo) * K / (hi - lo).  Almost every element gets there with one fp32
+        // subtraction and one fused multiply-add, and no float <-> integer conversion (those run at a quarter of the fp32
+        // rate): with 2^S the largest power of two such that K * 2^S <= 2^22 and r = K * 2^S / (hi - lo) rounded once,
+        //     t = fma(x - lo, r, 2^23)
+        // lies in [2^23, 2^24), where floats are the integers, so the low 23 bits of t ARE n = round((x - lo) * r), and
+        // |n - q * 2^S| <= 1: the subtraction (lo is exact in fp32) and r are each within 2^-24 relative, together at most
+        // q * 2^S * 2^-23 <= 1/2, and the fma rounds once to an integer, at most 1/2.  So wherever n mod 2^S is neither
+        // 0, 1, 2^S - 2 nor 2^S - 1, n >> S is the exact bin.  The other elements (4 in 2^S: about one in ten thousand for
+        // a hundred bins, and always the channel's minimum and maximum) take the fp64 division.  r = 0 gives n = 0 and sends
+        // every element of a channel there (a constant channel, or a range whose lower end is not an fp16 value).
+        const int S = 22 - (32 - __clz(bins - 1));                            // bins >= 2
+        const unsigned int frac_mask = (1u << S) - 1u;
         float lf[8], rf[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const double l = lo[c0 + k];
             const double rng = __dsub_rn(hi[c0 + k], l);
             lf[k] = (float)l;
-            rf[k] = (rng > 0.0 && (double)lf[k] == l) ? (float)((double)bins / rng) : 0.f;
+            rf[k] = (rng > 0.0 && (double)lf[k] == l) ? (float)(((double)bins / rng) * (double)(1 << S)) : 0.f;
+            if (!(rf[k] <= 0x1p60f)) rf[k] = 0.f;                            // (a range so small that r overflows: exact path)
         }
-        // "further than eps from an integer" as one compare: |frac - 1/2| < 1/2 - eps
-        const float half_band = 0.5f - (float)bins * 0x1p-21f;
-        unsigned int *cnt_k[8];                                            // this thread's eight counter rows
+        uint32_t cnt_k[8];                                                 // this thread's counter of bin 0 for each of its channels
 #pragma unroll
-        for (int k = 0; k < 8; ++k) cnt_k[k] = s_cnt + (cl + k) * bins;
+        for (int k = 0; k < 8; ++k)
+            cnt_k[k] = (uint32_t)__cvta_generic_to_shared(s_cnt + ((k * bins) * 8 + tx) * R + (ty & (R - 1)));
+        const unsigned int last_bin = (unsigned int)(bins - 1);
         auto count_row = [&](const uint4 &v) {
             const __half2 *h2 = reinterpret_cast<const __half2 *>(&v);
 #pragma unroll
@@ -203,31 +218,76 @@ __global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restr
                 for (int e = 0; e < 2; ++e) {
                     const int k = 2 * k2 + e;
                     const float xf = e ? xf2.y : xf2.x;
-                    const float qf = (xf - lf[k]) * rf[k];
-                    int b = __float2int_rd(qf);
-                    const float fr = qf - (float)b;
-                    if (!(fabsf(fr - 0.5f) < half_band)) b = histogram_exact_bin(xf, c0 + k, bins, lo, hi);
-                    atomicAdd(cnt_k[k] + b, 1u);
+                    const unsigned int n = __float_as_uint(fmaf(xf - lf[k], rf[k], 8388608.f)) - 0x4B000000u;
+                    // (the clamp keeps the index inside the counter row whatever the input, e.g. a NaN)
+                    unsigned int b = min(n >> S, last_bin);
+                    if (((n + 2u) & frac_mask) < 4u) b = (unsigned int)histogram_exact_bin(xf, c0 + k, bins, lo, hi);
+                    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(cnt_k[k] + (uint32_t)(32 * R) * b) : "memory");
                 }
             }
         };
-        // four rows per thread in flight
-        int r = r_begin + ty;
-        for (; r + 96 < r_end; r += 128) {
-            uint4 v[4];
+        // This thread's rows are r_begin + ty + 32 * i, i < n.  Loads and counting must overlap, and with 80 registers per thread
+        // (three CTAs per SM) there is no room for a second set of rows in registers: every thread keeps kHistAhead of its own
+        // 16-byte pieces in flight into a private slot ring in shared memory (asynchronous copies, one group per row; no
+        // other thread touches the slots, so no barrier is needed).
+        const int n = (r_end - r_begin - ty + 31) / 32;
+        const __half *xcol = X + (long)(r_begin + ty) * ldx + c0;
+        uint4 *ring = reinterpret_cast<uint4 *>(s_cnt + 64 * R * bins) + threadIdx.x;      // slot j of this thread: ring[256 * j]
+        const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+        // (one slot more than rows in flight: the slot being refilled is the one read an iteration ago, whose values are used up)
+        int wr = 0;
+        auto fetch = [&](int i) {
+            if (i < n)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + (uint32_t)(wr * 4096)),
+                             "l"(xcol + (long)i * 32 * ldx)
+                             : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");          // (an empty group past the end keeps the count in step)
+            wr = wr == kHistAhead ? 0 : wr + 1;
+        };
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = __ldg(reinterpret_cast<const uint4 *>(X + (long)(r + 32 * u) * ldx + c0));
-#pragma unroll
-            for (int u = 0; u < 4; ++u) count_row(v[u]);
+        for (int i = 0; i < kHistAhead; ++i) fetch(i);
+        int rd = 0;
+        for (int i = 0; i < n; ++i) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(kHistAhead - 1) : "memory");
+            const uint4 v = ring[256 * rd];
+            rd = rd == kHistAhead ? 0 : rd + 1;
+            fetch(i + kHistAhead);
+            count_row(v);
         }
-        for (; r < r_end; r += 32) count_row(__ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0)));
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
     for (int i = threadIdx.x; i < 64 * bins; i += 256) {
-        int c = blockIdx.x * 64 + i / bins;
-        unsigned int n = s_cnt[i];
-        if (c < C && n) atomicAdd(&counts[(long)c * bins + (i % bins)], n);
+        const int cc = i / bins, b = i - cc * bins;                        // channel of this CTA, bin
+        const int c = blockIdx.x * 64 + cc;
+        const unsigned int *src = s_cnt + (((cc & 7) * bins + b) * 8 + (cc >> 3)) * R;
+        unsigned int n = 0;
+#pragma unroll
+        for (int rep = 0; rep < R; ++rep) n += src[rep];
+        if (c < C && n) atomicAdd(&counts[(long)c * bins + b], n);
     }
+}
+
+// Counter replicas for a bin count: as many as keep three CTAs on an SM (about 75 KB each), none beyond.
+inline esp_status_t launch_histogram(const __half *X, int T, int C, long ldx, int splits, int bins, const double *lo,
+                                     const double *hi, unsigned int *counts, cudaStream_t stream) {
+    const size_t per_replica = sizeof(unsigned int) * 64 * (size_t)bins;
+    const size_t ring = (size_t)(kHistAhead + 1) * 256 * 16;
+    const int R = per_replica * 4 + ring <= 75 * 1024 ? 4 : per_replica * 2 + ring <= 75 * 1024 ? 2 : 1;
+    const size_t smem = per_replica * R + ring;
+    const dim3 grid(ceil_div(C, 64), splits);
+    const int rows = ceil_div(T, splits);
+    if (R == 4) {
+        ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        histogram_kernel<4><<<grid, 256, smem, stream>>>(X, T, C, ldx, rows, bins, lo, hi, counts);
+    } else if (R == 2) {
+        ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        histogram_kernel<2><<<grid, 256, smem, stream>>>(X, T, C, ldx, rows, bins, lo, hi, counts);
+    } else {
+        ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        histogram_kernel<1><<<grid, 256, smem, stream>>>(X, T, C, ldx, rows, bins, lo, hi, counts);
+    }
+    return ESP_OK;
 }
 
 // IR_c = -sum_k p_k ln p_k (Eq. 1, bins in index order, empty bins skipped) and s_c = IR_c + alpha*AM_c (Eq. 3).
@@ -487,7 +547,11 @@ __device__ void lbs_slot_prepare(const uint16_t *__restrict__ Wt, long ldt, cons
 __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, const double (&sc_fixed)[4], int k, int cx,
                                      double sx, const uint32_t *__restrict__ pk, const unsigned long long *s_B) {
     const int lane = threadIdx.x & 31;
-    long long Ax = 0, D[4] = {0, 0, 0, 0};
+    // Per-lane sums of |w| are kept as doubles: every term is a multiple of 2^-24 below 2^16 and a lane adds fewer than
+    // 2^11 of them, so every partial sum is a multiple of 2^-24 below 2^27 -- 51 bits, exact in fp64 -- and equals the
+    // integer sum of group_value_warp once scaled by 2^24.  (One conversion and one predicated add per term instead of the
+    // shifts, selects and 64-bit adds of the integer form: this loop is bound by instruction issue.)
+    double Ax = 0.0, D0 = 0.0, D1 = 0.0, D2 = 0.0, D3 = 0.0;
     const uint16_t *col = Wt + (long)cx * ldt;
     // The decision "is the candidate ahead of f2" is the fp64 comparison of |w_x| * s_x with |w_f2| * s_f2.  Its fp32 image
     // (exact |w|, scores rounded once, one rounded multiply: each product within 2^-23 relative of its fp64 counterpart)
@@ -502,28 +566,30 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const uint16_t hx = reinterpret_cast<const uint16_t *>(&vx)[e];
-            const int f2 = (int)(pkv[e] >> 16);
-            const uint16_t hf = (uint16_t)(pkv[e] & 0xFFFFu);
-            const float px = __half2float(__ushort_as_half(hx)) * sx32;      // (hx, hf hold magnitudes: the sign bit is clear)
-            const float pf = __half2float(__ushort_as_half(hf)) * (f2 == 0 ? s32[0] : f2 == 1 ? s32[1] : f2 == 2 ? s32[2] : s32[3]);
+            const uint32_t rec = pkv[e];
+            const uint16_t hf = (uint16_t)(rec & 0xFFFFu);
+            const bool f2_odd = (rec & 0x10000u) != 0, f2_high = (rec & 0x20000u) != 0;
+            const float wx = __half2float(__ushort_as_half(hx));           // (hx, hf hold magnitudes: the sign bit is clear)
+            const float wf = __half2float(__ushort_as_half(hf));
+            const float sf32 = f2_high ? (f2_odd ? s32[3] : s32[2]) : (f2_odd ? s32[1] : s32[0]);
+            const float px = wx * sx32, pf = wf * sf32;
             const float big = fmaxf(fabsf(px), fabsf(pf));                 // (scores may be negative when the caller supplies them)
-            const float margin = big * 0x1p-21f;
-            const bool normal = big >= 0x1p-100f;                           // below, fp32 products lose relative accuracy
-            bool kept;
-            if (normal && px - pf > margin) {
-                kept = true;
-            } else if (normal && pf - px > margin) {
-                kept = false;
-            } else {
+            const float diff = px - pf;
+            bool kept = diff > 0.f;
+            // undecided in fp32: closer than the margin, or so small that fp32 products lose relative accuracy
+            if (!(fabsf(diff) > big * 0x1p-21f && big >= 0x1p-100f)) {
+                const int f2 = (int)(rec >> 16);
                 const double sf = f2 == 0 ? sc_fixed[0] : f2 == 1 ? sc_fixed[1] : f2 == 2 ? sc_fixed[2] : sc_fixed[3];
                 const double xx = __dmul_rn(half_bits_abs_to_double(hx), sx);
                 const double xf = __dmul_rn(half_bits_abs_to_double(hf), sf);
                 kept = metric_ahead(xx, k, xf, f2);
             }
-            const long long wf = kept ? half_bits_abs_fixed(hf) : 0;
-            Ax += kept ? half_bits_abs_fixed(hx) : 0;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) D[q] += (q == f2) ? wf : 0;
+            if (kept) {
+                const double wfd = (double)wf;
+                Ax = __dadd_rn(Ax, (double)wx);
+                if (f2_high) { if (f2_odd) D3 = __dadd_rn(D3, wfd); else D2 = __dadd_rn(D2, wfd); }
+                else { if (f2_odd) D1 = __dadd_rn(D1, wfd); else D0 = __dadd_rn(D0, wfd); }
+            }
         }
     };
     // the column comes from L2: four 16-byte loads per lane are in flight before the first is used
@@ -536,16 +602,19 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
         for (int u = 0; u < 4; ++u) rows8(v[u], j + u * 256);
     }
     for (; j < ldt; j += 256) rows8(__ldg(reinterpret_cast<const uint4 *>(col + j)), j);
+    long long Axi = __double2ll_rn(__dmul_rn(Ax, 0x1p24));                  // exact: see above
+    long long D[4] = {__double2ll_rn(__dmul_rn(D0, 0x1p24)), __double2ll_rn(__dmul_rn(D1, 0x1p24)),
+                      __double2ll_rn(__dmul_rn(D2, 0x1p24)), __double2ll_rn(__dmul_rn(D3, 0x1p24))};
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        Ax += __shfl_xor_sync(0xFFFFFFFFu, Ax, off);
+        Axi += __shfl_xor_sync(0xFFFFFFFFu, Axi, off);
 #pragma unroll
         for (int q = 0; q < 4; ++q) D[q] += __shfl_xor_sync(0xFFFFFFFFu, D[q], off);
     }
     double t[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-        const long long A = (q == k) ? Ax : (long long)s_B[q] - D[q];
+        const long long A = (q == k) ? Axi : (long long)s_B[q] - D[q];
         const double sq = (q == k) ? sx : sc_fixed[q];
         t[q] = __dmul_rn(sq, __dmul_rn(__ll2double_rn(A), 0x1p-24));
     }
@@ -1016,10 +1085,7 @@ esp_status_t launch_calib_histogram(const CalibState &c, const __half *X, int T,
     esp_status_t st = device_info(&di);
     if (st != ESP_OK) return st;
     const int hsplits = pick_splits(T, ceil_div(C, 64), di.sm_count);
-    const size_t hsmem = sizeof(unsigned int) * 64 * (size_t)bins;
-    ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem));
-    histogram_kernel<<<dim3(ceil_div(C, 64), hsplits), 256, hsmem, stream>>>(X, T, C, ldx, ceil_div(T, hsplits), bins, c.lo, c.hi,
-                                                                             c.counts);
+    if (launch_histogram(X, T, C, ldx, hsplits, bins, c.lo, c.hi, c.counts, stream) != ESP_OK) return ESP_ERR_CUDA;
     ESP_CUDA_OK(cudaGetLastError());
     return ESP_OK;
 }
@@ -1067,11 +1133,7 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
         // K2
         ESP_CUDA_OK(cudaMemsetAsync(w.counts, 0, sizeof(unsigned int) * (size_t)C * o.bins, stream));
         const int hsplits = pick_splits(T, ceil_div(C, 64), di.sm_count);
-        const int rows2 = ceil_div(T, hsplits);
-        const size_t hsmem = sizeof(unsigned int) * 64 * (size_t)o.bins;
-        ESP_CUDA_OK(cudaFuncSetAttribute(histogram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem));
-        histogram_kernel<<<dim3(ceil_div(C, 64), hsplits), 256, hsmem, stream>>>(Xcal, T, C, ldx, rows2, o.bins, w.lo,
-                                                                                 w.hi, w.counts);
+        if (launch_histogram(Xcal, T, C, ldx, hsplits, o.bins, w.lo, w.hi, w.counts, stream) != ESP_OK) return ESP_ERR_CUDA;
         entropy_score_kernel<<<cblocks, cthreads, 0, stream>>>(C, T, o.bins, w.counts, w.norm, o.alpha, o.use_entropy,
                                                                o.use_norm, o.score_override, w.entropy, w.score);
     } else {

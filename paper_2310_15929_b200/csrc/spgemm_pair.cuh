@@ -43,10 +43,14 @@
 // every CTA pushes its fp32 partial rows to the CTA of the same pair rank in the owning slice (16-byte asynchronous remote
 // stores), which adds the slices in slice order.
 //
-// QUAD = true (tiled form only) puts two pairs on the same 512 features and neighbouring token tiles into one cluster of
-// four; each CTA fetches one of its two weight tiles and hands a copy to the other pair through distributed shared memory.
-// Correct and bit-identical to the plain form, but slower on every shape measured (the hand-over chain does not fit a
-// three-slot ring): kept for comparison, never planned.
+// SHARE != 0 (tiled form only) puts two pairs on the same 512 features and neighbouring token tiles into one cluster of
+// four, so that a weight tile leaves L2 once per two token tiles.  kShareHandOver: each CTA fetches one of its two weight
+// tiles and hands a copy to the other pair through distributed shared memory.  kShareReplicate: each CTA fetches one weight
+// tile with a load that the memory system delivers to both pairs (that load is supplied by another translation unit, see
+// SharedTileLoad below).  Both are bit-identical to the plain form and both are slower on every shape measured: the
+// hand-over chain does not fit a three-slot ring, a cluster of four leaves 16 of 148 SMs idle (33 clusters fit), and in
+// either form every SM still takes in the same 68 KB per step -- what limits the kernel is that intake, not the bytes
+// leaving L2.  Kept for comparison, never planned.
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -317,11 +321,23 @@ __device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *a
     return false;
 }
 
-template <int NA, int TN, bool TILED, bool QUAD = false>
+// How the two pairs of a four-CTA cluster share weight tiles (SHARE below): not at all (clusters of two), by a hand-over
+// through distributed shared memory, or by a load that the memory system delivers to both pairs at once.  The last form's
+// load instruction is not in this file: the translation unit that builds that form specialises this struct with
+//   static __device__ void rows(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar, uint16_t cta_mask)
+// (box of whole 1024-byte rows to offset `dst` of every CTA of the mask, bytes reported to the barrier at `bar`'s offset in the
+// even CTA of each destination's pair).
+constexpr int kShareNone = 0, kShareHandOver = 1, kShareReplicate = 2;
+template <int SHARE>
+struct SharedTileLoad;
+
+template <int NA, int TN, bool TILED, int SHARE = kShareNone>
 __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const GemmParams p, const __grid_constant__ CUtensorMap wmap,
                                                                       const __grid_constant__ CUtensorMap xmap) {
     using L = PairCfg<NA, TN>;
     constexpr int STAGES = L::kStages;
+    constexpr bool QUAD = SHARE != kShareNone;                            // clusters of four: two pairs on the same features
+    constexpr bool REPL = SHARE == kShareReplicate;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -332,7 +348,7 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
     const uint32_t recv_bar = bar_base + 8u * 26;
     auto wland = [&](int s) { return bar_base + 8u * (16 + s); };     // QUAD: this CTA's own weight tile of the stage has landed
     auto wrecv = [&](int s) { return bar_base + 8u * (32 + s); };     // QUAD: the partner's weight tile has arrived here
-    static_assert(!QUAD || (TILED && NA == 2), "the four-CTA form exists for the tiled two-accumulator kernel");
+    static_assert(SHARE == kShareNone || (TILED && NA == 2), "the four-CTA forms exist for the tiled two-accumulator kernel");
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kBarOff + 8 * 25);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L::kBarOff + 8 * 25 + 4);
 
@@ -390,11 +406,13 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // and reports its bytes to it directly (rank 1's own `full` barriers stay unused).
             // QUAD: the X copies of both CTAs (if the pair has tokens) + from each CTA of the pair one "my own weight tile
             // has landed" and one "the partner's tile has arrived"; a slot is free once BOTH pairs' MMAs are done with it.
+            // REPL: the X copies of both CTAs (if the pair has tokens) + the four weight-tile copies of the cluster, each of
+            // which reports to both pairs' leaders.
             mbar_init(full(s), QUAD ? (has_tokens ? 6u : 4u)
                                : TILED ? 2u + (uint32_t)n_present + (uint32_t)n_present_peer
                                        : (uint32_t)kPairProducers + (uint32_t)n_present + (rank == 0 ? 1u : 0u));
             mbar_init(empty(s), QUAD ? 2 : 1);
-            if (QUAD) { mbar_init(wland(s), 1); mbar_init(wrecv(s), 1); }
+            if (QUAD && !REPL) { mbar_init(wland(s), 1); mbar_init(wrecv(s), 1); }
         }
         mbar_init(accum_bar, 1);
         mbar_init(recv_bar, 1);
@@ -500,10 +518,52 @@ __global__ void __launch_bounds__(kPairThreads, 1) spgemm_pair_kernel(const Gemm
             // ---- copy issuers: lane 0 of warp 2 + s * (NA + 1) + kind feeds ring slot s with weight tile `kind` (< NA) or
             // with the X image (kind == NA); it meets every phase of its slot's `empty` barrier.  The other lanes wait at
             // the vote below without polling.
-            constexpr int kCopies = QUAD ? 4 : NA + 1;
+            constexpr int kCopies = REPL ? 2 : QUAD ? 4 : NA + 1;
             static_assert(kCopies * STAGES <= 15, "one issuing warp per copy of the ring; warp 17 polls the accumulator barrier");
             const int iw = warp - 2;
-            if (QUAD && lane == 0 && iw < kCopies * STAGES) {
+            if constexpr (REPL) if (lane == 0 && iw < kCopies * STAGES) {
+                // ---- two lanes per ring slot: 0 fetches ONE weight tile (accumulator `qpair`'s, for this CTA's pair rank)
+                // into this CTA and into the CTA of the same pair rank in the other pair with a single load; 1 fetches the X
+                // image.  Both of this CTA's weight tiles of a stage therefore arrive from two loads, one of its own and one
+                // of the other pair's, and a tile crosses the L2 -> SM path once per two token tiles.  A slot may be refilled
+                // once BOTH pairs' MMAs are done with it (`empty` takes both commits), since the load writes into both.
+                const int s = iw / kCopies, role = iw % kCopies;
+                const int a_own = qpair;
+                const uint32_t full_own = map_to_rank(full(s), lead), full_other = map_to_rank(full(s), lead ^ 2u);
+                constexpr int kRowBytes = 1024;
+                if (role == 0) {
+                    const int row_step = kTileBytes / kRowBytes;
+                    const int row0 = ftile[a_own] * p.k_tiles * row_step;
+                    const uint32_t dst = sbase + s * L::kStage + a_own * kTileBytes;
+                    const uint16_t both = (uint16_t)((1u << rank) | (1u << (rank + 2u)));
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                        if (present[a_own]) {
+                            mbar_arrive_expect_tx_cluster(full_own, kTileBytes);
+                            mbar_arrive_expect_tx_cluster(full_other, kTileBytes);
+                            SharedTileLoad<SHARE>::rows(dst, &wmap, row0 + it * row_step, full_own, both);
+                        } else {
+                            mbar_arrive_remote(full_own);
+                            mbar_arrive_remote(full_other);
+                        }
+                    }
+                } else if (has_tokens) {
+                    const uint32_t *xflag = p.xflags + (size_t)(ttile * 2 + rank) * p.k_tiles;
+                    const int row_step = L::kXStage / kRowBytes;
+                    const int row0 = (int)((ttile * 2 + rank) * p.k_tiles) * row_step;
+                    const uint32_t dst = sbase + s * L::kStage + L::kWStage;
+                    for (int it = s; it < nk; it += STAGES) {
+                        const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                        if (!xflag_wait(xflag + it, abort_flag)) { alive = false; break; }
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                        if (!mbar_wait_1t(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                        mbar_arrive_expect_tx_cluster(full_own, (uint32_t)L::kXStage);
+                        tma_rows_pair(dst, &xmap, row0 + it * row_step, full_own);
+                    }
+                }
+            }
+            if (QUAD && !REPL && lane == 0 && iw < kCopies * STAGES) {
                 // ---- four lanes per ring slot: 0 fetches this CTA's share of the weight tiles, 1 the X image, 2 hands the
                 // fetched tile on to the partner CTA once it has landed, 3 reports the tile received from the partner
                 const int s = iw / kCopies, role = iw % kCopies;
@@ -917,7 +977,7 @@ esp_status_t launch_pair(const GemmParams &p, bool dependent, cudaStream_t strea
 template <int TN>
 esp_status_t launch_quad(const GemmParams &p, bool dependent, cudaStream_t stream) {
     using L = PairCfg<2, TN>;
-    auto kern = spgemm_pair_kernel<2, TN, true, true>;
+    auto kern = spgemm_pair_kernel<2, TN, true, kShareHandOver>;
     ESP_CUDA_OK(ensure_dynamic_smem((const void *)kern, L::kTotal));
     const int f_tiles = (p.N + 127) / 128, t_tiles = (p.M + TN - 1) / TN;
     cudaLaunchConfig_t cfg = {};

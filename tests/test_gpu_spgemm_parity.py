@@ -8,6 +8,7 @@ in the binade above the exact value), and the fp32 sum itself differs from the e
 partial additions, bounded here by 2^-16 * sum_k |w_k x_k| (the oracle forms that sum of magnitudes next to the product).
 """
 import math
+import os
 
 import numpy as np
 import pytest
@@ -229,6 +230,36 @@ def test_quad_kernel_shares_weight_tiles_between_two_pairs(M, N, K):
     bias = (g.standard_normal(N) * 2).astype(np.float16)
     Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=7, bias=bias, relu=True, static_weights=1), Yb)
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 200, 264), (520, 640, 1160), (1000, 1100, 520), (4100, 1536, 1160), (2048, 512, 4224)])
+def test_quad_multicast_kernel(M, N, K):
+    """The four-CTA form in which one load delivers a weight tile to both pairs of the cluster (the kernel of the optional
+    companion library).  Same MMAs in the same order as the pair kernel: identical bits -- with an odd number of token tiles
+    (the last cluster's second pair only fetches weights for the first), feature tiles beyond N, every tile width, both
+    layouts, a step count that is not a multiple of the ring depth."""
+    from paper_2310_15929_b200 import binding as b
+    from paper_2310_15929_b200.build import MC_SOURCE
+    if not b.esp_multicast_available():
+        # the companion's source is deliberately left out of multi-GPU runs; with the source present its absence is a fault
+        assert not os.path.exists(MC_SOURCE), "libesparse_mc.so is missing or does not load although its source is here"
+        pytest.skip("companion library left out of this run")
+    from tests.gpu_util import pack_on_gpu, spgemm
+    vals, meta, theta = pruned(M + N + K + 2, N, K)
+    g = np.random.default_rng(M + 2)
+    X = g.standard_normal((M, K)).astype(np.float16)
+    packed = pack_on_gpu(vals, meta)
+    Yref = ref_product(X, vals, meta, theta)
+    for tile in (240, 224, 192):
+        a = spgemm(X, packed, theta, N, channel_major=True, kernel=9, token_tile=tile, out_f32=True)
+        check(a, Yref, True)
+        assert np.array_equal(a, spgemm(X, packed, theta, N, channel_major=True, kernel=6, token_tile=tile, out_f32=True))
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=9), Yref)      # the planner's own tile
+    check(spgemm(X, packed, theta, N, kernel=9), Yref)                          # token-major X
+    bias = (g.standard_normal(N) * 2).astype(np.float16)
+    Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
+    check(spgemm(X, packed, theta, N, channel_major=True, kernel=9, bias=bias, relu=True, static_weights=1), Yb)
+    assert b.esp_last_device_status() == 0
 
 
 @pytest.mark.parametrize("M,N,K", [(300, 200, 264), (520, 640, 1160), (1000, 1100, 520), (4100, 1536, 1160), (2048, 512, 4224)])
