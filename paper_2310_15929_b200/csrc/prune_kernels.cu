@@ -209,8 +209,12 @@ __global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restr
         for (int k = 0; k < 8; ++k)
             cnt_k[k] = (uint32_t)__cvta_generic_to_shared(s_cnt + ((k * bins) * 8 + tx) * R + (ty & (R - 1)));
         const unsigned int last_bin = (unsigned int)(bins - 1);
+        // One branch per row of eight elements, not one per element: the eight estimates are formed first, together with the
+        // smallest distance-to-a-boundary code among them; only a row that holds an undecided element (about one row in a
+        // thousand) goes back over its elements.
         auto count_row = [&](const uint4 &v) {
             const __half2 *h2 = reinterpret_cast<const __half2 *>(&v);
+            unsigned int b[8], closest = 0xFFFFFFFFu;
 #pragma unroll
             for (int k2 = 0; k2 < 4; ++k2) {
                 const float2 xf2 = __half22float2(h2[k2]);
@@ -220,11 +224,20 @@ __global__ void __launch_bounds__(256, 3) histogram_kernel(const __half *__restr
                     const float xf = e ? xf2.y : xf2.x;
                     const unsigned int n = __float_as_uint(fmaf(xf - lf[k], rf[k], 8388608.f)) - 0x4B000000u;
                     // (the clamp keeps the index inside the counter row whatever the input, e.g. a NaN)
-                    unsigned int b = min(n >> S, last_bin);
-                    if (((n + 2u) & frac_mask) < 4u) b = (unsigned int)histogram_exact_bin(xf, c0 + k, bins, lo, hi);
-                    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(cnt_k[k] + (uint32_t)(32 * R) * b) : "memory");
+                    b[k] = min(n >> S, last_bin);
+                    closest = min(closest, (n + 2u) & frac_mask);
                 }
             }
+            if (closest < 4u) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float xf = __half2float(reinterpret_cast<const __half *>(&v)[k]);
+                    const unsigned int n = __float_as_uint(fmaf(xf - lf[k], rf[k], 8388608.f)) - 0x4B000000u;
+                    if (((n + 2u) & frac_mask) < 4u) b[k] = (unsigned int)histogram_exact_bin(xf, c0 + k, bins, lo, hi);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(cnt_k[k] + (uint32_t)(32 * R) * b[k]) : "memory");
         };
         // This thread's rows are r_begin + ty + 32 * i, i < n.  Loads and counting must overlap, and with 80 registers per thread
         // (three CTAs per SM) there is no room for a second set of rows in registers: every thread keeps kHistAhead of its own

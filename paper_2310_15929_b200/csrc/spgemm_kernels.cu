@@ -1077,8 +1077,12 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
                 const long clusters = f_pairs * ceil_div(M, tn);
                 const double mma = 4.0 * tn, copy = (36864.0 + (tn > 128 ? 32768.0 : 16384.0)) / 70.0;
                 // per wave: the channel steps (both terms show in the measured step time), an epilogue that grows with the
-                // tile (about ten steps' worth at 240 tokens) and a fixed set-up
-                const double cost = (double)ceil_div(clusters, per_wave) * (0.5 * (mma + copy) * k_tiles + 40.0 * tn + 2000.0);
+                // tile (about ten steps' worth at 240 tokens) and a fixed set-up.  Waves: a grid of up to two waves runs as
+                // whole waves (equal tiles end together); over many waves the clusters drift apart and the last, partial wave
+                // costs less and less of a whole one (measured at 4.4 waves: already closer to the fractional count).
+                const double w = (double)clusters / (double)per_wave, whole = (double)ceil_div(clusters, per_wave);
+                const double waves = w <= 2.0 ? whole : w + (whole - w) * (2.0 / w);
+                const double cost = waves * (0.5 * (mma + copy) * k_tiles + 40.0 * tn + 2000.0);
                 if (best < 0.0 || cost < best) { best = cost; bn = tn; }
             }
         }
