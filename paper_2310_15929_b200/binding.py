@@ -20,7 +20,7 @@ ESP_X_TOKEN_MAJOR, ESP_X_CHANNEL_MAJOR = 0, 1
 ESP_OUT_F16, ESP_OUT_F32 = 0, 1
 ESP_ACT_NONE, ESP_ACT_RELU = 0, 1
 ESP_KERNEL_AUTO, ESP_KERNEL_GATHER, ESP_KERNEL_TMA, ESP_KERNEL_STREAM, ESP_KERNEL_PAIR, ESP_KERNEL_PAIR_TILED = 0, 1, 2, 4, 5, 6
-ESP_KERNEL_QUAD_TILED, ESP_KERNEL_PAIR_PERSIST, ESP_KERNEL_QUAD_MULTICAST = 7, 8, 9
+ESP_KERNEL_QUAD_TILED, ESP_KERNEL_PAIR_PERSIST, ESP_KERNEL_QUAD_MULTICAST, ESP_KERNEL_STREAM_IMAGES = 7, 8, 9, 10
 
 
 class esp_prune_opts(ctypes.Structure):

@@ -48,7 +48,7 @@ static esp_status_t check_gemm_opts(const esp_gemm_opts *o) {
     if (o->force_kernel != ESP_KERNEL_AUTO && o->force_kernel != ESP_KERNEL_GATHER && o->force_kernel != ESP_KERNEL_TMA &&
         o->force_kernel != ESP_KERNEL_STREAM && o->force_kernel != ESP_KERNEL_PAIR && o->force_kernel != ESP_KERNEL_PAIR_TILED &&
         o->force_kernel != ESP_KERNEL_QUAD_TILED && o->force_kernel != ESP_KERNEL_PAIR_PERSIST &&
-        o->force_kernel != ESP_KERNEL_QUAD_MULTICAST)
+        o->force_kernel != ESP_KERNEL_QUAD_MULTICAST && o->force_kernel != ESP_KERNEL_STREAM_IMAGES)
         return ESP_ERR_INVALID_ARG;
     if (o->static_weights != 0 && o->static_weights != 1) return ESP_ERR_INVALID_ARG;
     if (o->activation != ESP_ACT_NONE && o->activation != ESP_ACT_RELU) return ESP_ERR_INVALID_ARG;
@@ -325,6 +325,11 @@ esp_status_t esp_spgemm_tune(const void *X, int M, int K, long ldx, const void *
             for (int tile : {240, 224, 192}) cands.push_back({ESP_KERNEL_PAIR_PERSIST, tile, 1, 0});      // never planned, sometimes ahead
     }
     if (M <= 1024) {
+        for (int tile : {64, 128})
+            for (int split = 1; split <= 8; ++split) {
+                if (tile >= 2 * M && tile > 64) continue;
+                cands.push_back({ESP_KERNEL_STREAM_IMAGES, tile, split, 0});
+            }
         for (int tile : {16, 32, 64, 128, 256}) {
             if (tile < M && tile < 256 && (M + tile - 1) / tile > 8) continue;      // many narrow token tiles: never the best
             if (tile >= 2 * M && tile > 16) continue;

@@ -253,6 +253,22 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     return false;
 }
 
+// Bounded wait for an image flag (set by a CTA of the tiling pass that is resident before this kernel can start).
+__device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v == 1u) return true;
+        if (i > 8) {
+            if (*abort_flag) return false;
+            __nanosleep(128);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
+    return false;
+}
+
 constexpr int kMaxStages = 12;
 constexpr int kPermRing = 16;        // stages of permutation entries kept ahead in shared memory
 

@@ -527,11 +527,16 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     constexpr uint32_t kTmemCols = tmem_cols_for(BN);
     const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
     const int prefetch = min(stages, nk);
+    // Image form (BN >= 64, a workspace): a tiling pass has written the permuted, swizzled X operand of every (64-token
+    // block, channel step) into the workspace; a stage's X is then one bulk copy per token block instead of 16-byte row
+    // copies from every producer thread (which are limited to one 32-byte sector per clock per SM).
+    const bool imaged = BN >= 64 && p.ximg != nullptr;
     const uint32_t rank = (split > 1) ? cluster_ctarank() : 0u;
     const int owned = max(0, min(cnt4, BN - (int)rank * cnt4));      // rows of this tile that this CTA finishes
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(full(s), L::kProd + 1); mbar_init(empty(s), 1); }
+        // gather form: every X producer thread + the weight-tile copy; image form: the weight-tile copy + the X image copies
+        for (int s = 0; s < stages; ++s) { mbar_init(full(s), imaged ? 2u : (uint32_t)L::kProd + 1u); mbar_init(empty(s), 1); }
         mbar_init(accum_bar, 1);
         mbar_init(recv_bar, 1);
         *abort_flag = 0;
@@ -549,7 +554,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    if (warp >= 2 && warp < 6) {
+    if (warp >= 2 && warp < 6 && !imaged) {
         // permutation entries of the first stages, all loads in flight together (the X addresses depend on them)
         const int g = threadIdx.x - 64;
         int pre[kPermRing];
@@ -615,6 +620,39 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
         const bool ring_refill = nk > kPermRing;                      // long K-slices: keep the ring kPermRing stages ahead
         bool alive = true;
         int refill = -1;
+        if (imaged) {
+            // ---- image form: lane 0 of producer warp q feeds the ring slots s = q, q + 4, ...: the weight tile (beyond the
+            // start-up ones) and the X images of the tile's 64-token blocks, each a bulk copy.  A slot always has the same
+            // feeder, which therefore waits for the slot's `empty` phases one after the other (a thread that ran two phases
+            // ahead of a barrier would see the older phase of the same parity as complete).  The images are written by
+            // the tiling pass this kernel is a programmatic dependent of; a raised flag also says that everything before
+            // that pass is complete (its CTAs waited for it), so Y may be written once any flag has been seen.
+            const int q = warp - 2;
+            const int h0 = (int)blockIdx.y * L::kTokBlocks;                              // first 64-token block of this tile
+            const int n_blocks = min(L::kTokBlocks, 2 * ((p.M + 127) / 128) - h0);      // (the pass writes whole 128-token pairs)
+            if (q < 4 && lane == 0) {
+                for (int it = 0; it < nk; ++it) {
+                    const int s = it % stages;
+                    if ((s & 3) != q) continue;
+                    const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                    const int kt = kt_begin + it;
+                    bool seen = true;
+                    for (int tb = 0; tb < n_blocks; ++tb) seen = seen && xflag_wait(p.xflags + (size_t)(h0 + tb) * p.k_tiles + kt, abort_flag);
+                    if (!seen) { alive = false; break; }
+                    asm volatile("fence.proxy.async;" ::: "memory");   // the pass's generic-proxy writes, just acquired -> this thread's bulk read
+                    if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { alive = false; break; }
+                    if (it >= prefetch) {
+                        mbar_arrive_expect_tx(full(s), kTileBytes);
+                        bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
+                    }
+                    mbar_arrive_expect_tx(full(s), (uint32_t)(n_blocks * L::kBlockBytes));
+                    for (int tb = 0; tb < n_blocks; ++tb)
+                        bulk_load(sbase + s * L::kStage + kTileBytes + tb * L::kBlockBytes,
+                                  p.ximg + ((size_t)(h0 + tb) * p.k_tiles + kt) * L::kBlockBytes, L::kBlockBytes, full(s));
+                }
+            }
+            if (nk == 0) grid_dependency_wait();                      // (no flag to see: wait for the stream order itself)
+        } else {
         grid_dependency_wait();                                       // X may come from the preceding kernel
         for (int it = 0; it < nk; ++it) {
             const int s = it % stages;
@@ -661,12 +699,21 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
                 bulk_load(sbase + s * L::kStage, w_src + (long)it * kTileBytes, kTileBytes, full(s));
             }
         }
+        }
         // ---- epilogue.  One K-slice: the first four producer warps (one quarter of the accumulator lanes each) stage
         // the tile in shared memory and store it.  Several: every producer warp pushes partial rows to their owners
         // (warp w reads lane quarter w % 4 and the 16-column pieces (w - 2) / 4, + kProd / 128, ...), then finishes the rows
         // this CTA owns.
         const int quarter = warp & 3;
         const int f_local = quarter * 32 + lane;
+        if (imaged) {
+            // Almost every producer thread has been idle since the start: one of them polls the accumulator barrier, the
+            // others sleep on a named barrier (hundreds of lanes polling through the main loop slow the CTA's other
+            // barrier operations down).
+            if (warp == 6 && lane == 0 && nk > 0) (void)mbar_wait(accum_bar, 0, abort_flag);
+            __syncwarp();
+            asm volatile("bar.sync 1, %0;" ::"n"(L::kProd) : "memory");
+        }
         if (split == 1) {
             if (warp < 6) {
             const bool ok = __all_sync(0xFFFFFFFFu, alive && (nk == 0 || mbar_wait(accum_bar, 0, abort_flag)));   // warp-uniform
@@ -999,7 +1046,7 @@ static size_t ximg_bytes(int M, int K, int tn) {
 size_t gemm_workspace_min_bytes(int M, int K, const esp_gemm_opts &o) { return transpose_bytes(M, K, o); }
 size_t gemm_workspace_bytes(int M, int K, const esp_gemm_opts &o) {
     size_t n = transpose_bytes(M, K, o);
-    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || (o.force_kernel == ESP_KERNEL_AUTO && M > 64 && o.split_k <= 4) || o.force_kernel == ESP_KERNEL_QUAD_TILED ||
+    const bool pair_possible = o.force_kernel == ESP_KERNEL_PAIR_TILED || o.force_kernel == ESP_KERNEL_STREAM_IMAGES || (o.force_kernel == ESP_KERNEL_AUTO && M > 16) || o.force_kernel == ESP_KERNEL_QUAD_TILED ||
                                o.force_kernel == ESP_KERNEL_PAIR_PERSIST || o.force_kernel == ESP_KERNEL_QUAD_MULTICAST;
     if (pair_possible) {
         size_t img = 0;
@@ -1051,6 +1098,7 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
         else if (o.force_kernel == ESP_KERNEL_PAIR_PERSIST) g.kernel = ESP_KERNEL_PAIR_PERSIST;
         else if (o.force_kernel == ESP_KERNEL_QUAD_MULTICAST) g.kernel = ESP_KERNEL_QUAD_MULTICAST;
         else if (o.force_kernel == ESP_KERNEL_STREAM) g.kernel = ESP_KERNEL_STREAM;
+        else if (o.force_kernel == ESP_KERNEL_STREAM_IMAGES) g.kernel = ESP_KERNEL_STREAM_IMAGES;
         else {
             // The pair kernel takes every M > 64; a requested token tile or slice count that only the streaming kernel has
             // (tiles below 128 tokens, more than four slices, slices of a 256-token tile) goes there.
@@ -1061,6 +1109,24 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
             const long pairs128 = (long)ceil_div(f_tiles, 4) * ceil_div(M, 128);
             const bool pair = !stream_only && (M > 256 || (M > 64 && pairs128 >= 20));
             g.kernel = pair ? ESP_KERNEL_PAIR : ESP_KERNEL_STREAM;
+            // 17..256 tokens on a large weight: the streaming kernel fed from X images.  Its row gather limits the
+            // streaming kernel once the X tile is a good part of a stage; the images cost one more (small) launch, which pays
+            // from about 40 M weight elements (measured, gather form -> image form: 36864 x 9216 at 32 / 64 tokens
+            // 78 -> 67 / 118 -> 68 us; 9216 x 9216 at 64 / 128 tokens 41 -> 28 / 47 -> 37 us; but 9216 x 9216 at 32 tokens
+            // 22.5 -> 28.4, 4096 x 4096 at 128 tokens 15.0 -> 17.1).  It also replaces the pair kernel's gather form where that
+            // would run K-slices at 129..256 tokens (9216 x 9216 at 256 tokens: 95 -> 55 us).
+            const long weight = (long)N * K;
+            const bool images_room = workspace_bytes >= transpose_bytes(M, K, o) + ximg_bytes(M, K, 128);
+            if (images_room && bn == 0 && o.split_k <= 8 && M > 16 && M <= 256) {
+                const long per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
+                if (!pair) {
+                    const bool pays = M <= 32 ? weight >= 200000000L : M <= 64 ? (f_tiles >= 64 || weight >= 64000000L) : weight >= 40000000L;
+                    if (pays) { g.kernel = ESP_KERNEL_STREAM_IMAGES; bn = (M > 128 && weight >= 64000000L) ? 128 : 64; }
+                } else if (M > 128 && o.split_k == 0 && weight >= 80000000L && per_wave / pairs128 >= 2) {
+                    g.kernel = ESP_KERNEL_STREAM_IMAGES;
+                    bn = 128;
+                }
+            }
         }
     }
     const bool wide_only = g.kernel == ESP_KERNEL_QUAD_TILED || g.kernel == ESP_KERNEL_PAIR_PERSIST ||
@@ -1120,14 +1186,15 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
             if ((long)f_tiles * ceil_div(M, narrow) * std::min(k_tiles, 8) <= 2L * di.sm_count) { bn = narrow; break; }
         }
     }
-    if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
+    if ((g.kernel == ESP_KERNEL_TMA || g.kernel == ESP_KERNEL_STREAM_IMAGES) && bn < 64) bn = 64;
+    if (g.kernel == ESP_KERNEL_STREAM_IMAGES && workspace_bytes < transpose_bytes(M, K, o) + ximg_bytes(M, K, 128)) return ESP_ERR_WORKSPACE;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
     g.stages = 4;
     const int t_tiles = ceil_div(M, bn);
     const long tiles = (long)f_tiles * t_tiles;
     auto no_empty_slice = [&](int split) { return (long)ceil_div(k_tiles, split) * (split - 1) < k_tiles; };
-    if (g.kernel == ESP_KERNEL_STREAM) {
+    if (g.kernel == ESP_KERNEL_STREAM || g.kernel == ESP_KERNEL_STREAM_IMAGES) {
         // Pick K-slices and CTAs per SM so that, if possible, the whole grid is resident at once and each CTA
         // has a short chain of tiles: cost ~ waves x (tiles per CTA + fixed start-up and reduction time).
         const size_t per_stage = (size_t)kTileBytes + 256 * (size_t)bn;
@@ -1162,7 +1229,7 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
                 // wide token tiles are bound by their X gather, which CTAs sharing an SM share: a step costs as many
                 // times more as CTAs of one wave sit on an SM
                 const long in_wave = ctas < cap ? ctas : cap;
-                const double share = bn >= 64 ? (double)((in_wave + di.sm_count - 1) / di.sm_count) : 1.0;
+                const double share = (bn >= 64 && g.kernel == ESP_KERNEL_STREAM) ? (double)((in_wave + di.sm_count - 1) / di.sm_count) : 1.0;
                 double cost = (double)waves * (kts * share + 2.0 + bn / 32.0) + (split > 1 ? 0.25 + 0.05 * split : 0.0) + 0.01 * r;
                 // with static_weights consecutive launches overlap on an SM: prefer leaving room for a CTA of the next one
                 // (not when every CTA has an SM of its own anyway: a deeper ring is then free, measured 16.0 -> 12.6 us on
@@ -1318,7 +1385,7 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
         }
     }
     if (plan.kernel != ESP_KERNEL_GATHER) {
-        if (!p.x_channel_major && plan.kernel != ESP_KERNEL_PAIR_TILED) {
+        if (!p.x_channel_major && plan.kernel != ESP_KERNEL_PAIR_TILED && plan.kernel != ESP_KERNEL_STREAM_IMAGES) {
             // token-major input: transposed (not permuted) copy into the caller's workspace
             const long ldt = transposed_ld(M);
             if (!workspace || workspace_bytes < (size_t)K * ldt * 2) return ESP_ERR_WORKSPACE;
@@ -1352,6 +1419,25 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
                 case 224: return launch_pair<2, 224>(p, dependent, stream);
                 case 240: return launch_pair<2, 240>(p, dependent, stream);
                 case 256: return launch_pair<1, 256>(p, dependent, stream);
+                default: return ESP_ERR_INVALID_ARG;
+            }
+        }
+        if (plan.kernel == ESP_KERNEL_STREAM_IMAGES) {
+            // the tiling pass writes the images of 64-token blocks (the 128-token pair kernel's format); the streaming kernel
+            // follows as its programmatic dependent and takes each image when its flag is up
+            const size_t off = transpose_bytes(M, K, o);
+            if (!workspace || workspace_bytes < off + ximg_bytes(M, K, 128)) return ESP_ERR_WORKSPACE;
+            uint8_t *img = reinterpret_cast<uint8_t *>(workspace) + off;
+            uint32_t *flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<128>(M, K));
+            p.ximg = img;
+            p.xflags = flags;
+            const esp_status_t st = p.x_channel_major ? launch_xtile<128>(p, img, flags, dependent, stream)
+                                                      : launch_xtile_tm<128>(p, reinterpret_cast<const uint16_t *>(X), ldx, img, flags, dependent, stream);
+            if (st != ESP_OK) return st;
+            switch (plan.token_tile) {
+                case 64: return launch_stream<64>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
+                case 128: return launch_stream<128>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
+                case 256: return launch_stream<256>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
                 default: return ESP_ERR_INVALID_ARG;
             }
         }
@@ -1391,7 +1477,9 @@ esp_status_t launch_spgemm_group(int count, const void *const *X, int M, int K, 
     const size_t tbytes = transpose_bytes(M, K, o);
     if (tbytes > 0 && (!workspace || workspace_bytes < tbytes * (size_t)count)) return ESP_ERR_UNSUPPORTED;
     GemmPlan plan;
-    esp_status_t st = plan_gemm(M, f_total * kTileFeat, K, o, workspace ? workspace_bytes : 0, &plan);
+    esp_gemm_opts og = o;                    // (a group shares one launch of the streaming kernel's gather form)
+    if (og.force_kernel == ESP_KERNEL_AUTO && M <= 64) og.force_kernel = ESP_KERNEL_STREAM;
+    esp_status_t st = plan_gemm(M, f_total * kTileFeat, K, og, workspace ? workspace_bytes : 0, &plan);
     if (st != ESP_OK) return st;
     if (plan.kernel != ESP_KERNEL_STREAM) return ESP_ERR_UNSUPPORTED;
     GemmGroup grp;

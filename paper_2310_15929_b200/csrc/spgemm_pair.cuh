@@ -305,22 +305,6 @@ __global__ void __launch_bounds__(256) xtile_tm_kernel(const uint16_t *__restric
             asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flags + (size_t)h * k_tiles + kt), "r"(1u) : "memory");
 }
 
-// Bounded wait for an image flag (set by a CTA of the tiling pass that is resident before this kernel can start).
-__device__ __forceinline__ bool xflag_wait(const uint32_t *flag, volatile int *abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        uint32_t v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-        if (v == 1u) return true;
-        if (i > 8) {
-            if (*abort_flag) return false;
-            __nanosleep(128);
-        }
-    }
-    *abort_flag = 1;
-    atomicExch(&g_device_status, (int)ESP_ERR_TIMEOUT);
-    return false;
-}
-
 // How the two pairs of a four-CTA cluster share weight tiles (SHARE below): not at all (clusters of two), by a hand-over
 // through distributed shared memory, or by a load that the memory system delivers to both pairs at once.  The last form's
 // load instruction is not in this file: the translation unit that builds that form specialises this struct with
