@@ -198,10 +198,11 @@ enum { ESP_KERNEL_AUTO = 0,
                                     its own, accumulators straight from registers to Y) runs under the next tile's
                                     first steps (token_tile 192, 224 or 240; same results bit for bit; within a few
                                     per cent of ESP_KERNEL_PAIR_TILED either way, so only esp_spgemm_tune picks it) */
-       ESP_KERNEL_STREAM_IMAGES = 10,/* ESP_KERNEL_STREAM for 64-token blocks and wider (token_tile 64, 128 or 256), fed like
+       ESP_KERNEL_STREAM_IMAGES = 10,/* ESP_KERNEL_STREAM for token_tile 32, 64, 128 or 256, fed like
                                     ESP_KERNEL_PAIR_TILED: a pass over X writes the permuted, swizzled operand images of every
-                                    (64-token block, channel step) into the workspace and a stage's X is one bulk copy per
-                                    block instead of 16-byte row copies; same results bit for bit; needs the workspace  */
+                                    (token block, channel step) into the workspace and a stage's X is one bulk copy per
+                                    block instead of 16-byte row copies; same results bit for bit; needs the workspace
+                                    (default for 17..256 tokens on large weights)                        */
        ESP_KERNEL_QUAD_MULTICAST = 9 };/* the cluster of ESP_KERNEL_QUAD_TILED with every weight tile delivered to
                                     both pairs by ONE tiled load (cluster multicast of the tensor memory unit) instead
                                     of a hand-over: token_tile 192, 224 or 240, same results bit for bit.  Its kernel

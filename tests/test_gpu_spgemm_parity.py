@@ -236,7 +236,7 @@ def test_quad_kernel_shares_weight_tiles_between_two_pairs(M, N, K):
 def test_streaming_kernel_fed_from_images(M, N, K):
     """The streaming kernel with its X operand brought in as ready-made images (one bulk copy per 64-token block and step)
     instead of gathered rows: the same MMAs and the same K-slice reduction as the gather form, so identical bits -- for
-    every tile width it has (64, 128, 256), one and several K-slices, ragged M (a last 64-token block that the tiling pass
+    every tile width it has (32, 64, 128, 256), one and several K-slices, ragged M (a last 64-token block that the tiling pass
     leaves partly or wholly to padding), feature tiles beyond N, both layouts, both output types, bias and ReLU."""
     from tests.gpu_util import pack_on_gpu, spgemm
     vals, meta, theta = pruned(M + N + K + 3, N, K)
@@ -244,7 +244,7 @@ def test_streaming_kernel_fed_from_images(M, N, K):
     X = g.standard_normal((M, K)).astype(np.float16)
     packed = pack_on_gpu(vals, meta)
     Yref = ref_product(X, vals, meta, theta)
-    for tile in (64, 128, 256):
+    for tile in (32, 64, 128, 256):
         for split in (1, 2, 3):
             a = spgemm(X, packed, theta, N, channel_major=True, kernel=10, token_tile=tile, split_k=split, out_f32=True)
             check(a, Yref, True)
@@ -252,7 +252,7 @@ def test_streaming_kernel_fed_from_images(M, N, K):
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=10), Yref)     # the planner's own tile and slices
     h = spgemm(X, packed, theta, N, kernel=10, static_weights=1)                 # token-major X: the transposing tiling pass
     check(h, Yref)
-    assert np.array_equal(h, spgemm(X, packed, theta, N, kernel=4, token_tile=0))
+    check(spgemm(X, packed, theta, N, kernel=10, token_tile=32), Yref)           # token-major X, 32-token tiles: transposed copy first
     bias = (g.standard_normal(N) * 2).astype(np.float16)
     Yb = _with_magnitudes(orc.layer_output(Yref, bias, True), Yref.S + np.abs(bias.astype(np.float64))[None, :])
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=10, bias=bias, relu=True, static_weights=1), Yb)
