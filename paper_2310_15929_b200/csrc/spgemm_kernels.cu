@@ -527,11 +527,11 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     constexpr uint32_t kTmemCols = tmem_cols_for(BN);
     const uint8_t *w_src = p.packed + ((long)ft * p.k_tiles + kt_begin) * kTileBytes;
     const int prefetch = min(stages, nk);
-    // Image form (BN >= 32, a workspace): a tiling pass has written the permuted, swizzled X operand of every (64-token
-    // block -- BN = 32: 32-token tile --, channel step) into the workspace; a stage's X is then one bulk copy per token
+    // Image form (a workspace): a tiling pass has written the permuted, swizzled X operand of every (64-token
+    // block -- BN < 64: token tile --, channel step) into the workspace; a stage's X is then one bulk copy per token
     // block instead of 16-byte row copies from every producer thread (which are limited to one 32-byte sector per clock
     // per SM).
-    const bool imaged = BN >= 32 && p.ximg != nullptr;
+    const bool imaged = p.ximg != nullptr;
     const uint32_t rank = (split > 1) ? cluster_ctarank() : 0u;
     const int owned = max(0, min(cnt4, BN - (int)rank * cnt4));      // rows of this tile that this CTA finishes
 
@@ -630,7 +630,7 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
             // that pass is complete (its CTAs waited for it), so Y may be written once any flag has been seen.
             const int q = warp - 2;
             const int h0 = (int)blockIdx.y * L::kTokBlocks;                              // first 64-token block of this tile
-            const int n_blocks = BN == 32 ? 1 : min(L::kTokBlocks, 2 * ((p.M + 127) / 128) - h0);   // (64-token blocks: the pass writes whole 128-token pairs)
+            const int n_blocks = BN < 64 ? 1 : min(L::kTokBlocks, 2 * ((p.M + 127) / 128) - h0);   // (64-token blocks: the pass writes whole 128-token pairs)
             if (q < 4 && lane == 0) {
                 for (int it = 0; it < nk; ++it) {
                     const int s = it % stages;
@@ -826,18 +826,22 @@ __global__ void __launch_bounds__(StreamCfg<BN>::kThreads) spgemm_stream_kernel(
     }
 }
 
-// X [K, ldx] channel-major -> the streaming kernel's X stages for 32-token tiles: image (t, kt) holds channels
-// perm[kt*128 .. +127] of tokens 32 t .. 32 t + 31 as [128 rows][64 bytes] with the 16-byte chunk c of row r stored at chunk
-// c ^ ((r >> 1) & 3) (the 64-byte swizzle the kernel's B descriptor names).  Rows beyond K and tokens beyond M are zero.
-// grid (token tiles, k_tiles), block 256: thread -> row tid >> 1, chunks 2 (tid & 1) and + 1.  Flags as in xtile_kernel:
-// lowered before the dependent launch may start, raised when the image is complete.
-__global__ void __launch_bounds__(256) xtile32_kernel(const uint16_t *__restrict__ X, long ldx, int M, int K,
-                                                      const int32_t *__restrict__ perm, uint8_t *__restrict__ img,
-                                                      uint32_t *__restrict__ flags, int k_tiles) {
+// X [K, ldx] channel-major -> the streaming kernel's X stages for 16- and 32-token tiles: image (t, kt) holds channels
+// perm[kt*128 .. +127] of tokens BN t .. BN t + BN - 1 as [128 rows][2 BN bytes] with the 16-byte chunk c of row r stored
+// at the chunk the kernel's B descriptor expects (64-byte swizzle for 32 tokens: c ^ ((r >> 1) & 3); 32-byte swizzle for 16:
+// c ^ ((r >> 2) & 1)).  Rows beyond K and tokens beyond M are zero.  grid (token tiles, k_tiles), block 256: thread -> row
+// and chunk(s).  Flags as in xtile_kernel: lowered before the dependent launch may start, raised when the image is complete.
+template <int BN>
+__global__ void __launch_bounds__(256) xtile_narrow_kernel(const uint16_t *__restrict__ X, long ldx, int M, int K,
+                                                           const int32_t *__restrict__ perm, uint8_t *__restrict__ img,
+                                                           uint32_t *__restrict__ flags, int k_tiles) {
+    using L = StreamCfg<BN>;
+    static_assert(BN == 16 || BN == 32, "narrow tiles");
+    constexpr int kPer = L::kChunks / 2;                                  // chunks per thread: 2 threads per row
     const int t = blockIdx.x, kt = blockIdx.y;
-    uint8_t *dst = img + ((size_t)t * k_tiles + kt) * 8192;
+    uint8_t *dst = img + ((size_t)t * k_tiles + kt) * L::kBlockBytes;
     uint32_t *flag = flags + (size_t)t * k_tiles + kt;
-    const int r = threadIdx.x >> 1, c0 = (threadIdx.x & 1) * 2;
+    const int r = threadIdx.x >> 1, c0 = (threadIdx.x & 1) * kPer;
     const int kpos = kt * kTileK + r;
     const int ch = kpos < K ? (perm ? __ldg(perm + kpos) : kpos) : -1;
     grid_dependency_wait();                  // X may be the preceding kernel's output; the images may still be read by it
@@ -848,8 +852,8 @@ __global__ void __launch_bounds__(256) xtile32_kernel(const uint16_t *__restrict
     __syncthreads();
     grid_launch_dependents();
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int cc = c0 + i, tok = t * 32 + cc * 8;
+    for (int i = 0; i < kPer; ++i) {
+        const int cc = c0 + i, tok = t * BN + cc * 8;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (ch >= 0 && tok < M) {
             const uint16_t *src = X + (long)ch * ldx + tok;
@@ -863,19 +867,21 @@ __global__ void __launch_bounds__(256) xtile32_kernel(const uint16_t *__restrict
                                e[6] | ((uint32_t)e[7] << 16));
             }
         }
-        *reinterpret_cast<uint4 *>(dst + r * 64 + ((cc ^ ((r >> 1) & 3)) << 4)) = v;
+        const int cs = cc ^ ((r >> L::kSwzShift) & (L::kChunks - 1));
+        *reinterpret_cast<uint4 *>(dst + r * L::kRowBytes + (cs << 4)) = v;
     }
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(1u) : "memory");
 }
-inline size_t xtile32_image_bytes(int M, int K) { return (size_t)((M + 31) / 32) * ((K + kTileK - 1) / kTileK) * 8192; }
-inline size_t xtile32_bytes(int M, int K) {    // images | one flag word per image
-    return xtile32_image_bytes(M, K) + align_up((size_t)((M + 31) / 32) * ((K + kTileK - 1) / kTileK) * 4, 256);
+inline size_t xtile_narrow_image_bytes(int M, int K, int bn) { return (size_t)((M + bn - 1) / bn) * ((K + kTileK - 1) / kTileK) * 256 * bn; }
+inline size_t xtile_narrow_bytes(int M, int K, int bn) {    // images | one flag word per image
+    return xtile_narrow_image_bytes(M, K, bn) + align_up((size_t)((M + bn - 1) / bn) * ((K + kTileK - 1) / kTileK) * 4, 256);
 }
-inline esp_status_t launch_xtile32(const GemmParams &p, uint8_t *img, uint32_t *flags, bool dependent, cudaStream_t stream) {
+template <int BN>
+esp_status_t launch_xtile_narrow(const GemmParams &p, uint8_t *img, uint32_t *flags, bool dependent, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.M + 31) / 32, p.k_tiles, 1);
+    cfg.gridDim = dim3((p.M + BN - 1) / BN, p.k_tiles, 1);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -883,8 +889,8 @@ inline esp_status_t launch_xtile32(const GemmParams &p, uint8_t *img, uint32_t *
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile32_kernel, reinterpret_cast<const uint16_t *>(p.X), p.ldx, p.M, p.K, p.perm, img, flags,
-                                   p.k_tiles));
+    ESP_CUDA_OK(cudaLaunchKernelEx(&cfg, xtile_narrow_kernel<BN>, reinterpret_cast<const uint16_t *>(p.X), p.ldx, p.M, p.K, p.perm, img,
+                                   flags, p.k_tiles));
     return ESP_OK;
 }
 
@@ -1251,7 +1257,6 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
         }
     }
     if (g.kernel == ESP_KERNEL_TMA && bn < 64) bn = 64;
-    if (g.kernel == ESP_KERNEL_STREAM_IMAGES && bn < 32) bn = 32;
     if (g.kernel == ESP_KERNEL_STREAM_IMAGES && workspace_bytes < transpose_bytes(M, K, o) + ximg_bytes(M, K, 128)) return ESP_ERR_WORKSPACE;
     if (bn != 16 && bn != 32 && bn != 64 && bn != 128 && bn != 256) return ESP_ERR_INVALID_ARG;
     g.token_tile = bn;
@@ -1493,13 +1498,18 @@ esp_status_t launch_spgemm(const __half *X, int M, int K, long ldx, const void *
             // follows as its programmatic dependent and takes each image when its flag is up
             const size_t off = transpose_bytes(M, K, o);
             uint8_t *img = reinterpret_cast<uint8_t *>(workspace) + off;
-            if (plan.token_tile == 32) {     // 32-token tiles: images of their own format, from channel-major X (transposed above if need be)
-                if (!workspace || workspace_bytes < off + xtile32_bytes(M, K)) return ESP_ERR_WORKSPACE;
-                uint32_t *flags32 = reinterpret_cast<uint32_t *>(img + xtile32_image_bytes(M, K));
+            if (plan.token_tile < 64) {      // narrow tiles: images of their own format, from channel-major X (transposed above if need be)
+                const int bn = plan.token_tile;
+                if (!workspace || workspace_bytes < off + xtile_narrow_bytes(M, K, bn)) return ESP_ERR_WORKSPACE;
+                uint32_t *flags_n = reinterpret_cast<uint32_t *>(img + xtile_narrow_image_bytes(M, K, bn));
                 p.ximg = img;
-                p.xflags = flags32;
-                const esp_status_t st32 = launch_xtile32(p, img, flags32, dependent, stream);
-                return st32 != ESP_OK ? st32 : launch_stream<32>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
+                p.xflags = flags_n;
+                if (bn == 32) {
+                    const esp_status_t st_n = launch_xtile_narrow<32>(p, img, flags_n, dependent, stream);
+                    return st_n != ESP_OK ? st_n : launch_stream<32>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
+                }
+                const esp_status_t st_n = launch_xtile_narrow<16>(p, img, flags_n, dependent, stream);
+                return st_n != ESP_OK ? st_n : launch_stream<16>(p, f_tiles, t_tiles, plan.split_k, plan.stages, true, stream);
             }
             if (!workspace || workspace_bytes < off + ximg_bytes(M, K, 128)) return ESP_ERR_WORKSPACE;
             uint32_t *flags = reinterpret_cast<uint32_t *>(img + xtile_image_bytes<128>(M, K));

@@ -232,11 +232,12 @@ def test_quad_kernel_shares_weight_tiles_between_two_pairs(M, N, K):
     check(spgemm(X, packed, theta, N, channel_major=True, kernel=7, bias=bias, relu=True, static_weights=1), Yb)
 
 
-@pytest.mark.parametrize("M,N,K", [(40, 200, 264), (64, 640, 1160), (100, 1100, 2056), (128, 384, 4224), (200, 256, 520), (300, 640, 1032)])
+@pytest.mark.parametrize("M,N,K", [(1, 384, 1160), (13, 256, 2056), (40, 200, 264), (64, 640, 1160), (100, 1100, 2056), (128, 384, 4224), (200, 256, 520),
+                                   (300, 640, 1032)])
 def test_streaming_kernel_fed_from_images(M, N, K):
     """The streaming kernel with its X operand brought in as ready-made images (one bulk copy per 64-token block and step)
     instead of gathered rows: the same MMAs and the same K-slice reduction as the gather form, so identical bits -- for
-    every tile width it has (32, 64, 128, 256), one and several K-slices, ragged M (a last 64-token block that the tiling pass
+    every tile width it has (16 to 256), one and several K-slices, ragged M (a last 64-token block that the tiling pass
     leaves partly or wholly to padding), feature tiles beyond N, both layouts, both output types, bias and ReLU."""
     from tests.gpu_util import pack_on_gpu, spgemm
     vals, meta, theta = pruned(M + N + K + 3, N, K)
@@ -244,7 +245,7 @@ def test_streaming_kernel_fed_from_images(M, N, K):
     X = g.standard_normal((M, K)).astype(np.float16)
     packed = pack_on_gpu(vals, meta)
     Yref = ref_product(X, vals, meta, theta)
-    for tile in (32, 64, 128, 256):
+    for tile in (16, 32, 64, 128, 256):
         for split in (1, 2, 3):
             a = spgemm(X, packed, theta, N, channel_major=True, kernel=10, token_tile=tile, split_k=split, out_f32=True)
             check(a, Yref, True)
