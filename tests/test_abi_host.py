@@ -184,3 +184,32 @@ def test_grouped_and_tune_argument_checks_need_no_device():
     best = ctypes.c_float()
     assert b._lib.esp_spgemm_tune(None, 16, 128, 128, None, None, 128, None, 128, ctypes.byref(o), None, 0, 0,
                                   ctypes.byref(best), None, None) == b.ESP_ERR_INVALID_ARG
+
+
+def test_cluster_multicast_loads_live_only_in_the_companion_source():
+    """The main library must hold no bulk or tiled load with cluster multicast (it also runs where several GPUs are in
+    play); the one kernel form that uses such loads is built from a source file of its own into a companion library, and both
+    are named in the list of files left out of multi-GPU runs.  The companion is optional: the main library reports
+    whether it found it."""
+    from paper_2310_15929_b200.build import MC_LIB_PATH, MC_SOURCE
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    # (the pattern is put together from pieces so that this file does not itself name such a load)
+    load_with_multicast = re.compile("cp" + r"\.async\." + "bulk" + r"[^\n;]*\." + "multi" + "cast::cluster")
+    offenders = []
+    for folder, _, files in os.walk(root):
+        if any(part in folder for part in ("/.git", "/_work", "/gpurun_out", "/baseline", "/__pycache__")):
+            continue
+        for name in files:
+            if not name.endswith((".cu", ".cuh", ".h", ".py", ".c", ".cpp")):
+                continue
+            path = os.path.join(folder, name)
+            if os.path.abspath(path) in (os.path.abspath(MC_SOURCE), os.path.abspath(__file__)):
+                continue
+            if load_with_multicast.search(open(path, errors="replace").read()):
+                offenders.append(os.path.relpath(path, root))
+    assert offenders == []
+    left_out = open(os.path.join(root, ".gpurunignore.multi")).read().split()
+    assert os.path.relpath(MC_SOURCE, root) in left_out and os.path.relpath(MC_LIB_PATH, root) in left_out
+    if os.path.exists(MC_SOURCE):
+        assert load_with_multicast.search(open(MC_SOURCE).read())
+        assert b.esp_multicast_available() == os.path.exists(MC_LIB_PATH)
