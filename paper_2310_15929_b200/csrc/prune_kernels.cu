@@ -31,9 +31,13 @@ __device__ __forceinline__ long long half_bits_abs_fixed(uint16_t h) {
 // K1: per-channel sum of squares (fp64), min and max over a slice of tokens.   Eq. 2 / range of Eq. 1.
 // grid (ceil(C/256), splits), block 256 = 32 channel-vectors of 8 x 8 token lanes.
 // --------------------------------------------------------------------------------------------------
+constexpr int kColAhead = 8;                                              // rows each thread keeps in flight
+constexpr int kColSmem = (kColAhead + 1) * 256 * 16;                      // the threads' load rings; >= the partial results after
+static_assert(kColSmem >= (int)(sizeof(double) * 8 * 257 + 2 * sizeof(float) * 8 * 257), "the reduction reuses the ring");
 __global__ void __launch_bounds__(256) colstats_kernel(const __half *__restrict__ X, int T, int C, long ldx,
                                                        int rows_per_split, double *__restrict__ part_sumsq,
                                                        float *__restrict__ part_min, float *__restrict__ part_max) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int c0 = (blockIdx.x * 32 + tx) * 8;
     const int r_begin = blockIdx.y * rows_per_split;
@@ -53,19 +57,38 @@ __global__ void __launch_bounds__(256) colstats_kernel(const __half *__restrict_
                 mx[k] = fmaxf(mx[k], f);
             }
         };
-        // rows in the same order as a plain loop (the order of the fp64 additions is part of the result), four loads in flight
-        int r = r_begin + ty;
-        for (; r + 24 < r_end; r += 32) {
-            uint4 v[4];
+        // Rows in the same order as a plain loop (the order of the fp64 additions is part of the result).  This thread's rows
+        // are r_begin + ty + 8 i, i < n; kColAhead of its 16-byte pieces are kept in flight through a private slot ring in
+        // shared memory (asynchronous copies, one group per row; one slot more than rows in flight, so the slot being
+        // refilled is the one read an iteration ago) -- the registers leave no room for that many rows.
+        const int n = (r_end - r_begin - ty + 7) / 8;
+        const __half *xcol = X + (long)(r_begin + ty) * ldx + c0;
+        uint4 *ring = reinterpret_cast<uint4 *>(s_dyn) + threadIdx.x;      // slot j of this thread: ring[256 * j]
+        const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+        int wr = 0;
+        auto fetch = [&](int i) {
+            if (i < n)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + (uint32_t)(wr * 4096)), "l"(xcol + (long)i * 8 * ldx)
+                             : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");          // (an empty group past the end keeps the count in step)
+            wr = wr == kColAhead ? 0 : wr + 1;
+        };
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = __ldg(reinterpret_cast<const uint4 *>(X + (long)(r + 8 * u) * ldx + c0));
-#pragma unroll
-            for (int u = 0; u < 4; ++u) add_row(v[u]);
+        for (int i = 0; i < kColAhead; ++i) fetch(i);
+        int rd = 0;
+        for (int i = 0; i < n; ++i) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(kColAhead - 1) : "memory");
+            const uint4 v = ring[256 * rd];
+            rd = rd == kColAhead ? 0 : rd + 1;
+            fetch(i + kColAhead);
+            add_row(v);
         }
-        for (; r < r_end; r += 8) add_row(__ldg(reinterpret_cast<const uint4 *>(X + (long)r * ldx + c0)));
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
-    __shared__ double s_acc[8][256 + 1];
-    __shared__ float s_mn[8][256 + 1], s_mx[8][256 + 1];
+    __syncthreads();                         // every thread is done with its ring: the buffer now holds the partial results
+    double (*s_acc)[256 + 1] = reinterpret_cast<double (*)[256 + 1]>(s_dyn);
+    float (*s_mn)[256 + 1] = reinterpret_cast<float (*)[256 + 1]>(s_dyn + sizeof(double) * 8 * 257);
+    float (*s_mx)[256 + 1] = reinterpret_cast<float (*)[256 + 1]>(s_dyn + sizeof(double) * 8 * 257 + sizeof(float) * 8 * 257);
 #pragma unroll
     for (int k = 0; k < 8; ++k) { s_acc[ty][tx * 8 + k] = acc[k]; s_mn[ty][tx * 8 + k] = mn[k]; s_mx[ty][tx * 8 + k] = mx[k]; }
     __syncthreads();
@@ -753,28 +776,45 @@ __global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restr
         if (tid == 0) { int t = pos2x[bi]; pos2x[bi] = pos2x[bj]; pos2x[bj] = t; }
         ++swaps;
         __syncthreads();
-        // refresh: this CTA's (group, slot) rows of the table; units 0 and 4 also the base value of their group
+        // Refresh.  Row (g, slot) of the table holds the values of group g with that slot replaced by each candidate, so it
+        // depends on g's OTHER three channels only: of the eight rows of the two touched groups, the two rows of the swapped
+        // slots themselves stay as they are, six need new values.  Their candidates are dealt in quarters, three of the 24
+        // quarters to each of the cluster's eight CTAs (a CTA prepares the per-row records of each row it has a share of);
+        // units 0 and 4 also recompute the base value of one group each.
         {
-            const int g = unit < 4 ? (bi >> 2) : (bj >> 2);
-            const int slot = unit & 3;
-            int ch[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) ch[k] = chan[pos2x[g * 4 + k]];
-            double sc[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) sc[k] = score[ch[k]];
-            if (slot == 0 && warp == 0) {
-                double v = group_value_warp(Wt, ldt, score, ch[0], ch[1], ch[2], ch[3]);
+            if ((unit == 0 || unit == 4) && warp == 0) {
+                const int g = unit == 0 ? (bi >> 2) : (bj >> 2);
+                double v = group_value_warp(Wt, ldt, score, chan[pos2x[g * 4]], chan[pos2x[g * 4 + 1]], chan[pos2x[g * 4 + 2]],
+                                            chan[pos2x[g * 4 + 3]]);
                 if (lane == 0) base[p0 / 4 + g] = v;
             }
-            if (tid < 4) s_B[tid] = 0;
-            __syncthreads();
-            lbs_slot_prepare(Wt, ldt, score, ch, slot, s_pk, s_B);
-            __syncthreads();
-            for (int x = warp; x < m; x += 16) {
-                const int cx = chan[x];
-                const double v = lbs_slot_candidate(Wt, ldt, sc, slot, cx, score[cx], s_pk, s_B);
-                if (lane == 0) tb[(g * 4 + slot) * kLbsMax + x] = v;
+            const int quarter_size = (m + 3) >> 2;
+            int prepared = -1;
+            for (int qq = 3 * unit; qq < 3 * unit + 3; ++qq) {
+                const int row = qq >> 2, quarter = qq & 3, which = row / 3;
+                int slot = row - 3 * which;                      // the (row mod 3)-th slot other than the swapped one
+                if (slot >= ((which ? bj : bi) & 3)) ++slot;
+                const int g = (which ? bj : bi) >> 2;
+                int ch[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) ch[k] = chan[pos2x[g * 4 + k]];
+                double sc[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) sc[k] = score[ch[k]];
+                if (row != prepared) {
+                    __syncthreads();                             // the previous row's records are no longer being read
+                    if (tid < 4) s_B[tid] = 0;
+                    __syncthreads();
+                    lbs_slot_prepare(Wt, ldt, score, ch, slot, s_pk, s_B);
+                    __syncthreads();
+                    prepared = row;
+                }
+                const int x_end = min(m, (quarter + 1) * quarter_size);
+                for (int x = quarter * quarter_size + warp; x < x_end; x += 16) {
+                    const int cx = chan[x];
+                    const double v = lbs_slot_candidate(Wt, ldt, sc, slot, cx, score[cx], s_pk, s_B);
+                    if (lane == 0) tb[(g * 4 + slot) * kLbsMax + x] = v;
+                }
             }
         }
         __threadfence();
@@ -1086,7 +1126,7 @@ esp_status_t launch_calib_reset(const CalibState &c, int C, int bins, cudaStream
 esp_status_t launch_calib_range(const CalibState &c, const __half *X, int T, int C, long ldx, cudaStream_t stream) {
     int splits = ceil_div(T, 256);
     if (splits > 64) splits = 64;
-    colstats_kernel<<<dim3(ceil_div(C, 256), splits), 256, 0, stream>>>(X, T, C, ldx, ceil_div(T, splits), c.part_sumsq, c.part_min,
+    colstats_kernel<<<dim3(ceil_div(C, 256), splits), 256, kColSmem, stream>>>(X, T, C, ldx, ceil_div(T, splits), c.part_sumsq, c.part_min,
                                                                        c.part_max);
     calib_merge_kernel<<<ceil_div(C, 256), 256, 0, stream>>>(C, splits, c.part_sumsq, c.part_min, c.part_max, c.sumsq, c.lo, c.hi);
     ESP_CUDA_OK(cudaGetLastError());
@@ -1138,7 +1178,7 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
     if (need_stats_pass && Xcal) {
         // K1
         const int rows1 = ceil_div(T, w.splits);
-        colstats_kernel<<<dim3(ceil_div(C, 256), w.splits), 256, 0, stream>>>(Xcal, T, C, ldx, rows1, w.part_sumsq,
+        colstats_kernel<<<dim3(ceil_div(C, 256), w.splits), 256, kColSmem, stream>>>(Xcal, T, C, ldx, rows1, w.part_sumsq,
                                                                              w.part_min, w.part_max);
         colstats_finish_kernel<<<cblocks, cthreads, 0, stream>>>(C, w.splits, w.part_sumsq, w.part_min, w.part_max,
                                                                  w.norm, w.lo, w.hi);
