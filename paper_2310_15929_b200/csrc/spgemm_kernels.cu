@@ -1228,7 +1228,9 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
         int split = 1;
         if (bn == 128) {
             const long pairs = f_pairs * ceil_div(M, 128);
-            split = o.split_k > 0 ? o.split_k : (int)std::min<long>(4, std::max<long>(1, per_wave / pairs));
+            // (beyond 256 tokens two slices at most: three ran far slower than two -- 4096 x 4096 at 384 tokens 46 against
+            // 30 us, 4096 x 11008 at 384 tokens 70 against 50 -- and four no faster)
+            split = o.split_k > 0 ? o.split_k : (int)std::min<long>(M > 256 ? 2 : 4, std::max<long>(1, per_wave / pairs));
             while (split > 1 && (k_tiles / split < 4 || (long)ceil_div(k_tiles, split) * (split - 1) >= k_tiles)) --split;
         } else if (o.split_k > 1) {
             return ESP_ERR_INVALID_ARG;

@@ -196,17 +196,15 @@ def test_cluster_multicast_loads_live_only_in_the_companion_source():
     # (the pattern is put together from pieces so that this file does not itself name such a load)
     load_with_multicast = re.compile("cp" + r"\.async\." + "bulk" + r"[^\n;]*\." + "multi" + "cast::cluster")
     offenders = []
-    for folder, _, files in os.walk(root):
-        if any(part in folder for part in ("/.git", "/_work", "/gpurun_out", "/baseline", "/__pycache__")):
+    sources = [os.path.join(root, n) for n in os.listdir(root) if n.endswith(".py")]
+    for top in ("paper_2310_15929_b200", "include", "oracle", "tests"):
+        for folder, _, files in os.walk(os.path.join(root, top)):
+            sources += [os.path.join(folder, n) for n in files if n.endswith((".cu", ".cuh", ".h", ".py", ".c", ".cpp"))]
+    for path in sources:
+        if os.path.abspath(path) in (os.path.abspath(MC_SOURCE), os.path.abspath(__file__)):
             continue
-        for name in files:
-            if not name.endswith((".cu", ".cuh", ".h", ".py", ".c", ".cpp")):
-                continue
-            path = os.path.join(folder, name)
-            if os.path.abspath(path) in (os.path.abspath(MC_SOURCE), os.path.abspath(__file__)):
-                continue
-            if load_with_multicast.search(open(path, errors="replace").read()):
-                offenders.append(os.path.relpath(path, root))
+        if load_with_multicast.search(open(path, errors="replace").read()):
+            offenders.append(os.path.relpath(path, root))
     assert offenders == []
     left_out = open(os.path.join(root, ".gpurunignore.multi")).read().split()
     assert os.path.relpath(MC_SOURCE, root) in left_out and os.path.relpath(MC_LIB_PATH, root) in left_out
