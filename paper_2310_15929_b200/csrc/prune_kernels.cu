@@ -864,51 +864,65 @@ __global__ void __launch_bounds__(256) select_compress_kernel(const __half *__re
                                                               const double *__restrict__ score,
                                                               const int32_t *__restrict__ theta,
                                                               __half *__restrict__ vals, uint8_t *__restrict__ meta,
-                                                              unsigned long long *__restrict__ counters) {
-    extern __shared__ uint16_t s_row[];
-    const int j = blockIdx.x;
-    const uint16_t *Wr = reinterpret_cast<const uint16_t *>(W) + (long)j * ldw;
-    for (int c = threadIdx.x * 8; c < C; c += 256 * 8)
-        *reinterpret_cast<uint4 *>(s_row + c) = __ldg(reinterpret_cast<const uint4 *>(Wr + c));
+                                                              unsigned long long *__restrict__ counters, int rows_per_cta) {
+    // A CTA takes rows_per_cta consecutive output rows into shared memory; a thread then reads the permutation and the
+    // scores of its eight positions ONCE and applies them to every one of those rows (with one row per CTA the two gathers
+    // were six times the bytes of the row itself).
+    extern __shared__ __align__(16) uint16_t s_rows[];                  // [rows_per_cta][C]
+    const int j0 = blockIdx.x * rows_per_cta;
+    const int nrows = min(rows_per_cta, No - j0);
+    const int chunks_per_row = C / 8;
+    for (int idx = threadIdx.x; idx < nrows * chunks_per_row; idx += 256) {
+        const int r = idx / chunks_per_row, c = (idx - r * chunks_per_row) * 8;
+        *reinterpret_cast<uint4 *>(s_rows + (size_t)r * C + c) =
+            __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(W) + (long)(j0 + r) * ldw + c));
+    }
     __syncthreads();
     unsigned int near = 0;
     for (int u = threadIdx.x; u < C / 8; u += 256) {
-        uint16_t out[4];
-        unsigned int byte = 0;
+        int ch[8];
+        double sc[8];
 #pragma unroll
-        for (int gg = 0; gg < 2; ++gg) {
-            uint16_t h[4];
-            double xi[4];
+        for (int k = 0; k < 8; ++k) { ch[k] = theta[u * 8 + k]; sc[k] = score[ch[k]]; }
+        for (int r = 0; r < nrows; ++r) {
+            const uint16_t *s_row = s_rows + (size_t)r * C;
+            const long j = j0 + r;
+            uint16_t out[4];
+            unsigned int byte = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                int c = theta[u * 8 + gg * 4 + k];
-                h[k] = s_row[c];
-                xi[k] = __dmul_rn(half_bits_abs_to_double(h[k]), score[c]);
-            }
-            int kept[2], nk = 0;
-            double second = 0.0, third = 0.0;
+            for (int gg = 0; gg < 2; ++gg) {
+                uint16_t h[4];
+                double xi[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                int ahead = 0;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (q == k) continue;
-                    ahead += (xi[q] > xi[k] || (xi[q] == xi[k] && q < k)) ? 1 : 0;
+                for (int k = 0; k < 4; ++k) {
+                    h[k] = s_row[ch[gg * 4 + k]];
+                    xi[k] = __dmul_rn(half_bits_abs_to_double(h[k]), sc[gg * 4 + k]);
                 }
-                if (ahead < 2) { if (nk < 2) kept[nk] = k; ++nk; }
-                if (ahead == 1) second = xi[k];
-                if (ahead == 2) third = xi[k];
+                int kept[2], nk = 0;
+                double second = 0.0, third = 0.0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    int ahead = 0;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (q == k) continue;
+                        ahead += (xi[q] > xi[k] || (xi[q] == xi[k] && q < k)) ? 1 : 0;
+                    }
+                    if (ahead < 2) { if (nk < 2) kept[nk] = k; ++nk; }
+                    if (ahead == 1) second = xi[k];
+                    if (ahead == 2) third = xi[k];
+                }
+                if (__dsub_rn(second, third) < __dmul_rn(1e-6, second)) ++near;
+                out[gg * 2 + 0] = h[kept[0]];
+                out[gg * 2 + 1] = h[kept[1]];
+                byte |= (unsigned int)(kept[0] | (kept[1] << 2)) << (4 * gg);
             }
-            if (__dsub_rn(second, third) < __dmul_rn(1e-6, second)) ++near;
-            out[gg * 2 + 0] = h[kept[0]];
-            out[gg * 2 + 1] = h[kept[1]];
-            byte |= (unsigned int)(kept[0] | (kept[1] << 2)) << (4 * gg);
+            uint2 packed;
+            packed.x = (unsigned int)out[0] | ((unsigned int)out[1] << 16);
+            packed.y = (unsigned int)out[2] | ((unsigned int)out[3] << 16);
+            *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(vals) + j * (C / 2) + u * 4) = packed;
+            meta[j * (C / 8) + u] = (uint8_t)byte;
         }
-        uint2 packed;
-        packed.x = (unsigned int)out[0] | ((unsigned int)out[1] << 16);
-        packed.y = (unsigned int)out[2] | ((unsigned int)out[3] << 16);
-        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(vals) + (long)j * (C / 2) + u * 4) = packed;
-        meta[(long)j * (C / 8) + u] = (uint8_t)byte;
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) near += __shfl_xor_sync(0xFFFFFFFFu, near, off);
@@ -1260,12 +1274,17 @@ esp_status_t launch_prune(const __half *W, int No, int C, long ldw, const __half
 
     // K6 + K7
     const size_t row_smem = sizeof(uint16_t) * (size_t)C;
-    ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_smem));
+    // rows per CTA of the 2:4 kernel: as many as fit about 96 KB of shared memory (two CTAs per SM), eight at most
+    // (and no more than leave the grid two CTAs per SM)
+    int sel_rows = (int)std::max<size_t>(1, std::min<size_t>(8, (96 * 1024) / row_smem));
+    sel_rows = std::max(1, std::min(sel_rows, No / (2 * std::max(1, di.sm_count))));
+    ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(row_smem * sel_rows)));
     if (o.m_group == 8) {
         ESP_CUDA_OK(cudaFuncSetAttribute(select_compress_48_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_smem));
         select_compress_48_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
     } else
-        select_compress_kernel<<<No, 256, row_smem, stream>>>(W, No, C, ldw, w.score, perm, vals, meta, w.counters);
+        select_compress_kernel<<<ceil_div(No, sel_rows), 256, row_smem * sel_rows, stream>>>(W, No, C, ldw, w.score, perm, vals, meta,
+                                                                                             w.counters, sel_rows);
     ESP_CUDA_OK(cudaGetLastError());
     if (packed) {
         st = launch_pack(vals, meta, No, C, packed, stream);
