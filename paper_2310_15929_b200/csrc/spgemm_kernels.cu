@@ -1189,7 +1189,7 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
             if (images_room && bn == 0 && o.split_k <= 8 && M > 16 && M <= 256) {
                 const long per_wave = di.sm_count / 2 > 0 ? di.sm_count / 2 : 1;
                 if (!pair) {
-                    const bool pays = M <= 32 ? weight >= 200000000L : M <= 64 ? (f_tiles >= 64 || weight >= 64000000L) : weight >= 40000000L;
+                    const bool pays = M <= 32 ? weight >= 200000000L : M <= 64 ? (f_tiles >= 64 || weight >= 64000000L) : M <= 128 ? weight >= 40000000L : weight >= 16000000L;
                     // (up to 32 tokens: 32-token images -- 36864 x 9216 at 32 tokens 67.5 -> 64.3 us, 9216 x 36864 76 -> 70)
                     if (pays) { g.kernel = ESP_KERNEL_STREAM_IMAGES; bn = M <= 32 ? 32 : (M > 128 && weight >= 64000000L) ? 128 : 64; }
                 } else if (M > 128 && o.split_k == 0 && weight >= 80000000L && per_wave / pairs128 >= 2) {
@@ -1236,11 +1236,14 @@ static esp_status_t plan_gemm_uncached(int M, int N, int K, const esp_gemm_opts 
             return ESP_ERR_INVALID_ARG;
         }
         // the tiled form needs room for the X images behind the transposed copy; without it the gather form runs.  Up to
-        // 256 tokens the gather form is taken anyway: one launch instead of two, and X is small.
+        // 128 tokens the gather form is taken anyway: one launch instead of two, and X is small.
         const bool room = bn != 256 && workspace_bytes >= transpose_bytes(M, K, o) + ximg_bytes(M, K, bn);
         if ((g.kernel == ESP_KERNEL_PAIR_TILED || wide_only) && !room) return ESP_ERR_WORKSPACE;
         if (wide_only && (bn == 128 || bn == 256)) return ESP_ERR_INVALID_ARG;
-        if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room && M > 256) g.kernel = ESP_KERNEL_PAIR_TILED;
+        // (129..256 tokens in one K-slice: the tiled form too -- 11008 x 4096 at 256 tokens 37.4 -> 33.4 us, 13824 x 5120
+        // 47.2 -> 41.6; with K-slices the gather form stays ahead there)
+        if (g.kernel == ESP_KERNEL_PAIR && o.force_kernel == ESP_KERNEL_AUTO && room && (M > 256 || (M > 128 && split == 1)))
+            g.kernel = ESP_KERNEL_PAIR_TILED;
         g.token_tile = bn;
         g.split_k = split;
         g.stages = 0;
