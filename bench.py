@@ -44,7 +44,7 @@ WORKLOAD = SMALL_WORKLOAD                  # the profile cases below run on this
 # Headline step: 4 x (8192 x 8192) + 2 x (22016 x 8192) + (8192 x 22016) at 8192 tokens.
 PREFILL_TRAFFIC_BYTES = 4 * 0.923e9 + 2 * 2.126e9 + 2.28e9
 # Decode step at one token: 4 x (9216 x 9216) + (36864 x 9216) + (9216 x 36864).
-DECODE_TRAFFIC_BYTES = 4 * 98.7e6 + 386.6e6 + 387.3e6
+DECODE_TRAFFIC_BYTES = 4 * 99.1e6 + 388.5e6 + 387.5e6
 # bounded sample of the headline workload that the CPU oracle's product is timed on
 CPU_ROWS, CPU_FEATURES = 256, 1024
 
