@@ -659,7 +659,7 @@ __device__ double lbs_slot_candidate(const uint16_t *__restrict__ Wt, long ldt, 
 
 // table[b][g][slot][x] = V(group g of block b with its slot replaced by block channel x); base[G] = V(g).
 // grid (nblocks * 64 * 4): one CTA per (block, group, slot); block 256 (8 warps); dynamic shared memory ldt * 4 bytes.
-__global__ void __launch_bounds__(256) lbs_table_kernel(const uint16_t *__restrict__ Wt, long ldt,
+__global__ void __launch_bounds__(256, 4) lbs_table_kernel(const uint16_t *__restrict__ Wt, long ldt,
                                                         const double *__restrict__ score,
                                                         const int32_t *__restrict__ theta0, int C, int lbs_block,
                                                         double *__restrict__ table, double *__restrict__ base) {
@@ -693,12 +693,15 @@ __global__ void __launch_bounds__(256) lbs_table_kernel(const uint16_t *__restri
     }
 }
 
+// (Two CTAs per SM, at 64 registers per thread with a few spills: one cluster of eight occupies eight SMs whatever its
+// CTAs need, only 15 such clusters fit 148 SMs, and a weight has 32 to 86 blocks -- the second CTA per SM halves the number
+// of waves, and the LLaMA-65B-shaped layer's producer went from 3.4 to 2.1 s.)
 // One cluster of 8 CTAs per block of positions: repeat { best cross-group swap by table lookup; apply if gain > 0;
 // refresh the two touched groups }.  Every CTA takes the same decision from the same table (no exchange needed), then
 // refreshes one of the 2 groups x 4 slots of table rows; a cluster barrier publishes the rows before the next
 // decision.  grid (nblocks * 8), cluster (8), block 512, dynamic shared memory ldt * 4 bytes.
 constexpr int kLbsCluster = 8;
-__global__ void __launch_bounds__(512) lbs_greedy_kernel(const uint16_t *__restrict__ Wt, long ldt,
+__global__ void __launch_bounds__(512, 2) lbs_greedy_kernel(const uint16_t *__restrict__ Wt, long ldt,
                                                           const double *__restrict__ score,
                                                           const int32_t *__restrict__ theta0, int C, int lbs_block,
                                                           int max_swaps, double *__restrict__ table,
